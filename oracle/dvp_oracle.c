@@ -1,0 +1,263 @@
+/*
+ * dvp_oracle.c -- TEST INFRASTRUCTURE, NOT A PRODUCT PATH.
+ *
+ * Plain, slow, fp64 CPU statement of what Dynamic Vocabulary Pruning computes
+ * per token row.  It exists so that the CUDA library can be checked against
+ * the paper's definitions; only the tests, the smoke check and the benchmark's
+ * CPU-baseline leg may call it.  It shares no code, header, table or constant
+ * with the CUDA path.
+ *
+ * Notation (one row = one state s): logits z in R^V, sampled token a,
+ * pruning threshold rho, L = ln(rho), upstream gradient g.
+ *
+ *   safe set      V_S = { k : pi(k) >= rho * max_j pi(j) }              (Def. 5.1)
+ *                     = { k : z_k >= max_j z_j + L }    (App. A, protocol 2; the
+ *                       listing prunes with a strict '<', so equality is kept)
+ *   coverage      Z   = sum_{k in V_S} pi(k)                            (Def. 5.2)
+ *   pruned policy pi^mp(a) = pi(a) / Z  if a in V_S, else 0             (Def. 5.2)
+ *   masked logits z_mp,k = z_k on V_S, -inf elsewhere (Sec. 5.5, exact -inf
+ *                 semantics; softmax(z_mp) = pi^mp by Prop. 5.6 part 1)
+ *   gradient      d log pi^mp(a) / d z_k = 1[k=a] - pi^mp(k) on V_S, 0 off it,
+ *                 with the set held fixed (Prop. 5.4, Prop. 5.6 part 2,
+ *                 App. A protocol 1); a outside V_S has weight zero
+ *                 (remark after Thm. 5.3), so its row of gradients is zero.
+ *   log-ratio     r = log pi^mp_train(a) - log pi^mp_infer(a)
+ *                 (sign of Delta in Thm. 4.1; App. A protocol 4)
+ *
+ * Every sum is a Neumaier-compensated fp64 sum taken in index order.
+ * Nothing here is blocked, fused or reordered.
+ */
+#include <math.h>
+#include <pthread.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_F32 0
+#define ORACLE_BF16 1
+#define ORACLE_F16 2
+
+/* ---- exact widening of stored logits to double ------------------------- */
+
+static double widen_f32(const void *p, int64_t i) {
+  return (double)((const float *)p)[i];
+}
+
+static double widen_bf16(const void *p, int64_t i) {
+  /* bfloat16 is the upper half of an IEEE binary32 */
+  uint32_t bits = ((uint32_t)((const uint16_t *)p)[i]) << 16;
+  float f;
+  memcpy(&f, &bits, sizeof f);
+  return (double)f;
+}
+
+static double widen_f16(const void *p, int64_t i) {
+  /* IEEE binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits */
+  uint16_t h = ((const uint16_t *)p)[i];
+  int sign = (h >> 15) & 1;
+  int e = (h >> 10) & 0x1f;
+  int f = h & 0x3ff;
+  double v;
+  if (e == 0)
+    v = ldexp((double)f, -24);
+  else if (e == 31)
+    v = f ? NAN : INFINITY;
+  else
+    v = ldexp((double)(f + 1024), e - 25);
+  return sign ? -v : v;
+}
+
+static double widen(const void *p, int dtype, int64_t i) {
+  if (dtype == ORACLE_BF16) return widen_bf16(p, i);
+  if (dtype == ORACLE_F16) return widen_f16(p, i);
+  return widen_f32(p, i);
+}
+
+/* ---- compensated accumulation ------------------------------------------ */
+
+typedef struct {
+  double sum, comp;
+} nsum;
+
+static void nsum_add(nsum *a, double x) {
+  double t = a->sum + x;
+  if (fabs(a->sum) >= fabs(x))
+    a->comp += (a->sum - t) + x;
+  else
+    a->comp += (x - t) + a->sum;
+  a->sum = t;
+}
+
+static double nsum_value(const nsum *a) { return a->sum + a->comp; }
+
+/* ---- one side (train or infer) of one row ------------------------------ */
+
+typedef struct {
+  double max;        /* m = max_k z_k                                        */
+  double lse;        /* ln sum_k e^{z_k}                                     */
+  double lse_safe;   /* ln sum_{k in V_S} e^{z_k}                            */
+  double log_cov;    /* ln Z = lse_safe - lse                                */
+  double logp;       /* ln pi(a)                                             */
+  double logp_mp;    /* ln pi^mp(a), -inf when a is pruned                   */
+  double sum_safe;   /* sum_{k in V_S} e^{z_k - m}                           */
+  double sum_safe_x; /* the same sum without the term k = a                  */
+  double tau;        /* m + L                                                */
+  int64_t count;     /* |V_S|                                                */
+  int32_t member;    /* 1 when a in V_S                                      */
+  int32_t pad_;
+} oracle_side;
+
+/*
+ * z: V doubles.  a < 0 means "no sampled token": the statistics of the row
+ * are still produced and the per-token fields are NaN / 0.
+ * mask (optional): V bytes, 1 where k is in the safe set.
+ */
+void dvp_oracle_side(const double *z, int64_t V, int64_t a, double log_rho,
+                     oracle_side *out, uint8_t *mask) {
+  double m = -INFINITY;
+  for (int64_t k = 0; k < V; ++k)
+    if (z[k] > m) m = z[k];
+  const double tau = m + log_rho;
+
+  nsum all = {0, 0}, safe = {0, 0}, safe_x = {0, 0};
+  int64_t n = 0;
+  for (int64_t k = 0; k < V; ++k) {
+    const double e = exp(z[k] - m);
+    const int keep = z[k] >= tau;
+    nsum_add(&all, e);
+    if (keep) {
+      nsum_add(&safe, e);
+      if (k != a) nsum_add(&safe_x, e);
+      ++n;
+    }
+    if (mask) mask[k] = (uint8_t)keep;
+  }
+  const double s = nsum_value(&all), s_safe = nsum_value(&safe);
+  out->max = m;
+  out->tau = tau;
+  out->lse = m + log(s);
+  out->lse_safe = m + log(s_safe);
+  out->log_cov = log(s_safe) - log(s);
+  out->sum_safe = s_safe;
+  out->sum_safe_x = nsum_value(&safe_x);
+  out->count = n;
+  if (a >= 0 && a < V) {
+    out->member = z[a] >= tau;
+    out->logp = (z[a] - m) - log(s);
+    out->logp_mp = out->member ? (z[a] - m) - log(s_safe) : -INFINITY;
+  } else {
+    out->member = 0;
+    out->logp = NAN;
+    out->logp_mp = NAN;
+  }
+}
+
+/*
+ * Gradient of g * log pi^mp(a) with respect to the V logits of the row, the
+ * safe set held fixed.  The k = a entry is g * (1 - pi^mp(a)) written as
+ * g * (sum over V_S without a) / (sum over V_S), which has no cancellation.
+ */
+void dvp_oracle_side_grad(const double *z, int64_t V, int64_t a, double g,
+                          const oracle_side *st, double *grad) {
+  if (a < 0 || a >= V || !st->member) {
+    for (int64_t k = 0; k < V; ++k) grad[k] = 0.0;
+    return;
+  }
+  for (int64_t k = 0; k < V; ++k) {
+    if (z[k] >= st->tau)
+      grad[k] = -g * exp(z[k] - st->lse_safe);
+    else
+      grad[k] = 0.0;
+  }
+  grad[a] = g * (st->sum_safe_x / st->sum_safe);
+}
+
+/*
+ * Per-token log-ratio r = ln pi^mp_train(a) - ln pi^mp_infer(a).
+ * a outside the training set: the importance ratio is zero (remark after
+ * Thm. 5.3), r = -inf whatever the inference side says.  a inside the
+ * training set but outside the inference set: r = +inf.
+ */
+double dvp_oracle_log_ratio(const oracle_side *tr, const oracle_side *inf) {
+  if (!tr->member) return -INFINITY;
+  if (!inf->member) return INFINITY;
+  return tr->logp_mp - inf->logp_mp;
+}
+
+/* ---- batch driver: rows are independent, split statically over threads -- */
+
+typedef struct {
+  /* inputs */
+  const void *train, *infer; /* [T, ld] stored logits; infer may be NULL   */
+  int32_t dtype;             /* ORACLE_F32 / ORACLE_BF16 / ORACLE_F16      */
+  int32_t want_mask;         /* fill mask_t / mask_i                        */
+  int64_t T, V, ld_train, ld_infer;
+  const int64_t *ids;        /* [T]                                         */
+  const double *upstream;    /* [T] or NULL                                 */
+  double rho;
+  /* outputs, each [T] unless noted, each may be NULL */
+  oracle_side *side_t, *side_i;
+  double *log_ratio;
+  double *grad;              /* [T, V] doubles or NULL                      */
+  uint8_t *mask_t, *mask_i;  /* [T, V] bytes                                */
+} oracle_batch;
+
+typedef struct {
+  const oracle_batch *b;
+  int64_t row0, row1;
+} oracle_job;
+
+static void *oracle_rows(void *arg) {
+  const oracle_job *job = (const oracle_job *)arg;
+  const oracle_batch *b = job->b;
+  const double log_rho = b->rho > 0.0 ? log(b->rho) : -INFINITY;
+  double *z = (double *)malloc(sizeof(double) * (size_t)b->V);
+  for (int64_t t = job->row0; t < job->row1; ++t) {
+    const int64_t a = b->ids ? b->ids[t] : -1;
+    oracle_side st, si;
+    for (int64_t k = 0; k < b->V; ++k)
+      z[k] = widen(b->train, b->dtype, t * b->ld_train + k);
+    dvp_oracle_side(z, b->V, a, log_rho, &st,
+                    b->want_mask && b->mask_t ? b->mask_t + t * b->V : NULL);
+    if (b->side_t) b->side_t[t] = st;
+    if (b->grad)
+      dvp_oracle_side_grad(z, b->V, a, b->upstream ? b->upstream[t] : 0.0, &st,
+                           b->grad + t * b->V);
+    if (b->infer) {
+      for (int64_t k = 0; k < b->V; ++k)
+        z[k] = widen(b->infer, b->dtype, t * b->ld_infer + k);
+      dvp_oracle_side(z, b->V, a, log_rho, &si,
+                      b->want_mask && b->mask_i ? b->mask_i + t * b->V : NULL);
+      if (b->side_i) b->side_i[t] = si;
+      if (b->log_ratio) b->log_ratio[t] = dvp_oracle_log_ratio(&st, &si);
+    }
+  }
+  free(z);
+  return NULL;
+}
+
+/* Returns the number of threads used. */
+int dvp_oracle_batch(const oracle_batch *b, int nthreads) {
+  if (nthreads < 1) nthreads = 1;
+  if (nthreads > b->T) nthreads = b->T > 0 ? (int)b->T : 1;
+  if (nthreads > 1024) nthreads = 1024;
+  oracle_job jobs[1024];
+  pthread_t tid[1024];
+  const int64_t per = (b->T + nthreads - 1) / nthreads;
+  for (int i = 0; i < nthreads; ++i) {
+    jobs[i].b = b;
+    jobs[i].row0 = per * i < b->T ? per * i : b->T;
+    jobs[i].row1 = per * (i + 1) < b->T ? per * (i + 1) : b->T;
+  }
+  if (nthreads == 1) {
+    oracle_rows(&jobs[0]);
+    return 1;
+  }
+  for (int i = 0; i < nthreads; ++i)
+    pthread_create(&tid[i], NULL, oracle_rows, &jobs[i]);
+  for (int i = 0; i < nthreads; ++i) pthread_join(tid[i], NULL);
+  return nthreads;
+}
+
+int dvp_oracle_sizeof_side(void) { return (int)sizeof(oracle_side); }
+int dvp_oracle_sizeof_batch(void) { return (int)sizeof(oracle_batch); }

@@ -1,0 +1,322 @@
+"""Pins for the fp64 oracle: it is checked against what the paper and the
+mathematics fix, never against itself.
+
+Each test names the passage of the paper it leans on.  A second implementation
+inside a test is always written a different way (probability space instead of
+logit space, a library log-softmax on -inf-masked logits, autograd, central
+differences, exact rational arithmetic where it applies).
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rows(rng, T, V, scale=3.0):
+    return rng.normal(size=(T, V)) * scale
+
+
+# --------------------------------------------------------------------------
+# Brute force in probability space (Def. 5.1 and Def. 5.2 as printed), tiny V,
+# extended precision, every token a enumerated.
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("rho", [0.5, 0.1, 1e-2, 1e-4])
+def test_bruteforce_probability_space_every_token(rho):
+    rng = np.random.default_rng(7)
+    ld = np.longdouble
+    for V in (2, 3, 5, 8, 12):
+        z = _rows(rng, 6, V, scale=2.5)
+        # keep clear of the threshold so both spaces decide alike
+        tau = z.max(1, keepdims=True) + math.log(rho)
+        assert np.abs(z - tau).min() > 1e-9
+        for a in range(V):
+            ids = np.full(6, a)
+            res = oracle.dvp_rows_f64(z, ids, rho, want_mask=True)
+            for t in range(6):
+                e = np.exp(z[t].astype(ld) - z[t].max().astype(ld))
+                pi = e / e.sum()
+                safe = pi >= ld(rho) * pi.max()                    # Def. 5.1
+                Z = pi[safe].sum()                                 # Def. 5.2
+                pi_mp = np.where(safe, pi / Z, ld(0))
+                assert abs(float(pi_mp.sum()) - 1.0) < 1e-15
+                assert np.array_equal(res.train.mask[t].astype(bool), safe)
+                assert res.train.count[t] == safe.sum()
+                assert res.train.member[t] == int(safe[a])
+                assert res.train.logp[t] == pytest.approx(float(np.log(pi[a])), abs=1e-12)
+                assert res.train.log_cov[t] == pytest.approx(float(np.log(Z)), abs=1e-12)
+                if safe[a]:
+                    assert res.train.logp_mp[t] == pytest.approx(float(np.log(pi_mp[a])), abs=1e-12)
+                else:
+                    assert res.train.logp_mp[t] == -np.inf
+                assert res.train.max[t] == z[t].max()
+
+
+def test_rho_zero_is_full_log_softmax():
+    """Every token satisfies pi >= 0: the limit rho -> 0 of Def. 5.1."""
+    rng = np.random.default_rng(1)
+    z = _rows(rng, 5, 301, scale=4.0)
+    ids = rng.integers(0, 301, size=5)
+    res = oracle.dvp_rows_f64(z, ids, 0.0, want_mask=True)
+    ref = torch.log_softmax(torch.from_numpy(z), dim=-1).numpy()
+    want = ref[np.arange(5), ids]
+    np.testing.assert_allclose(res.train.logp_mp, want, atol=1e-12, rtol=0)
+    np.testing.assert_allclose(res.train.logp, want, atol=1e-12, rtol=0)
+    assert (res.train.count == 301).all() and res.train.mask.all()
+    np.testing.assert_allclose(res.train.log_cov, 0.0, atol=1e-14)
+    lse = torch.logsumexp(torch.from_numpy(z), dim=-1).numpy()
+    np.testing.assert_allclose(res.train.lse, lse, atol=1e-12, rtol=0)
+    np.testing.assert_allclose(res.train.lse_safe, lse, atol=1e-12, rtol=0)
+
+
+def test_rho_one_keeps_exactly_the_argmax_ties():
+    z = np.array([[0.5, 2.0, -1.0, 2.0, 1.999999, 2.0],
+                  [3.0, 1.0, 0.0, -2.0, 2.9, 1.0]])
+    res = oracle.dvp_rows_f64(z, np.array([1, 0]), 1.0, want_mask=True)
+    assert res.train.mask.tolist() == [[0, 1, 0, 1, 0, 1], [1, 0, 0, 0, 0, 0]]
+    assert res.train.count.tolist() == [3, 1]
+    assert res.train.logp_mp[0] == pytest.approx(-math.log(3.0), abs=1e-15)
+    assert res.train.logp_mp[1] == pytest.approx(0.0, abs=1e-15)
+    # a token just under the maximum is pruned at rho = 1
+    res = oracle.dvp_rows_f64(z, np.array([4, 4]), 1.0)
+    assert res.train.member.tolist() == [0, 0]
+    assert np.isneginf(res.train.logp_mp).all()
+
+
+def test_threshold_tie_is_kept():
+    """Def. 5.1 uses >=, and the listing of App. A prunes with a strict <."""
+    L = math.log(0.25)
+    z = np.array([[4.0, 4.0 + L, np.nextafter(4.0 + L, -np.inf), 0.0]])
+    res = oracle.dvp_rows_f64(z, np.array([1]), 0.25, want_mask=True)
+    assert res.train.mask.tolist() == [[1, 1, 0, 0]]
+    assert res.train.member[0] == 1
+
+
+@pytest.mark.parametrize("rho", [1.0, 0.3, 1e-3, math.exp(-13), 1e-20, 0.0])
+def test_invariants(rho):
+    rng = np.random.default_rng(11)
+    z = _rows(rng, 40, 257, scale=5.0)
+    ids = rng.integers(0, 257, size=40)
+    res = oracle.dvp_rows_f64(z, ids, rho, want_mask=True)
+    s = res.train
+    amax = z.argmax(1)
+    assert s.mask[np.arange(40), amax].all()              # argmax is always safe
+    assert (s.count >= 1).all() and (s.count == s.mask.sum(1)).all()
+    assert (s.log_cov <= 1e-15).all()                     # Z <= 1
+    member = s.member.astype(bool)
+    assert (s.logp_mp[member] >= s.logp[member] - 1e-15).all()   # pi/Z >= pi
+    np.testing.assert_allclose(s.logp_mp[member], (s.logp - s.log_cov)[member], atol=1e-12)
+    assert np.isneginf(s.logp_mp[~member]).all()
+    # renormalised probabilities over the safe set sum to one
+    for t in range(40):
+        p = np.exp(z[t][s.mask[t].astype(bool)] - s.lse_safe[t])
+        assert math.fsum(p) == pytest.approx(1.0, abs=1e-13)
+        assert s.lse_safe[t] <= s.lse[t] + 1e-15
+
+
+@pytest.mark.parametrize("rho", [0.2, 1e-2, 1e-4])
+def test_masked_logit_policy_equivalence(rho):
+    """Prop. 5.6 part 1: softmax of the -inf-masked logits is pi^mp.  The mask
+    is built the way App. A builds it (max, + log rho, strict <), by torch."""
+    rng = np.random.default_rng(3)
+    z = torch.from_numpy(_rows(rng, 16, 500, scale=3.0))
+    thr = z.max(dim=-1, keepdim=True).values + math.log(rho)
+    z_mp = torch.where(z < thr, torch.tensor(-math.inf, dtype=z.dtype), z)
+    ref = torch.log_softmax(z_mp, dim=-1).numpy()
+    for a_kind in ("random", "argmax"):
+        ids = rng.integers(0, 500, size=16) if a_kind == "random" else z.numpy().argmax(1)
+        res = oracle.dvp_rows_f64(z.numpy(), ids, rho, want_mask=True)
+        want = ref[np.arange(16), ids]
+        np.testing.assert_allclose(res.train.logp_mp, want, atol=1e-12, rtol=0)
+        assert np.array_equal(res.train.mask.astype(bool), (z >= thr).numpy())
+
+
+@pytest.mark.parametrize("rho", [0.3, 1e-2, 1e-4])
+def test_gradient_matches_autograd_of_masked_log_softmax(rho):
+    """Prop. 5.6 part 2 / Prop. 5.4 with the set fixed (App. A protocol 1)."""
+    rng = np.random.default_rng(5)
+    T, V = 12, 200
+    z = torch.from_numpy(_rows(rng, T, V, scale=3.0)).requires_grad_(True)
+    g = torch.from_numpy(rng.normal(size=T))
+    ids_np = rng.integers(0, V, size=T)
+    ids_np[:4] = z.detach().numpy().argmax(1)[:4]
+    with torch.no_grad():
+        thr = z.max(dim=-1, keepdim=True).values + math.log(rho)
+        pruned = z < thr
+    z_mp = torch.where(pruned, torch.tensor(-math.inf, dtype=z.dtype), z)
+    logp = torch.log_softmax(z_mp, dim=-1)[torch.arange(T), torch.from_numpy(ids_np)]
+    member = torch.isfinite(logp)
+    (logp[member] * g[member]).sum().backward()
+    res = oracle.dvp_rows_f64(z.detach().numpy(), ids_np, rho, upstream=g.numpy())
+    np.testing.assert_allclose(res.grad, z.grad.numpy(), atol=1e-13, rtol=1e-12)
+    assert (res.grad[~member.numpy()] == 0).all()          # pruned token: zero row
+    assert member.numpy().sum() >= 4 and (~member.numpy()).sum() >= 1
+
+
+def test_gradient_central_differences_and_structure():
+    rng = np.random.default_rng(9)
+    T, V, rho, h = 6, 40, 5e-2, 1e-5
+    z = _rows(rng, T, V, scale=2.0)
+    tau = z.max(1, keepdims=True) + math.log(rho)
+    assert np.abs(z - tau).min() > 10 * h
+    ids = z.argsort(1)[:, -2]                               # second largest: a member
+    g = rng.normal(size=T)
+    res = oracle.dvp_rows_f64(z, ids, rho, upstream=g, want_mask=True)
+    mask = res.train.mask.astype(bool)
+
+    def logp_mp_frozen(zz, t):
+        zs = zz[mask[t]]
+        m = zs.max()
+        return zz[ids[t]] - (m + math.log(math.fsum(np.exp(zs - m))))
+
+    for t in range(T):
+        for k in range(V):
+            zp, zm = z[t].copy(), z[t].copy()
+            zp[k] += h
+            zm[k] -= h
+            fd = g[t] * (logp_mp_frozen(zp, t) - logp_mp_frozen(zm, t)) / (2 * h)
+            assert res.grad[t, k] == pytest.approx(fd, abs=2e-9)
+        assert (res.grad[t][~mask[t]] == 0).all()
+        assert math.fsum(res.grad[t]) == pytest.approx(0.0, abs=1e-14)
+        # the sampled entry is g (1 - pi^mp(a)), every other safe entry is -g pi^mp(k)
+        assert res.grad[t, ids[t]] == pytest.approx(g[t] * (1 - math.exp(res.train.logp_mp[t])), abs=1e-14)
+
+
+def test_single_element_safe_set_has_exactly_zero_gradient():
+    z = np.array([[50.0, 1.0, 0.0, -3.0]])
+    res = oracle.dvp_rows_f64(z, np.array([0]), 1e-3, upstream=np.array([2.0]))
+    assert res.train.count[0] == 1 and res.train.logp_mp[0] == 0.0
+    assert (res.grad == 0).all()
+
+
+def test_total_variation_equals_one_minus_coverage():
+    """Proof of Prop. 5.5: TV(pi^mp, pi) = 1 - Z, by the half-L1 definition."""
+    rng = np.random.default_rng(13)
+    z = _rows(rng, 20, 9, scale=2.0)
+    res = oracle.dvp_rows_f64(z, np.zeros(20, dtype=np.int64), 0.2, want_mask=True)
+    for t in range(20):
+        pi = np.exp(z[t] - z[t].max())
+        pi /= pi.sum()
+        safe = res.train.mask[t].astype(bool)
+        pi_mp = np.where(safe, pi / pi[safe].sum(), 0.0)
+        tv = 0.5 * np.abs(pi_mp - pi).sum()
+        assert tv == pytest.approx(1.0 - math.exp(res.train.log_cov[t]), abs=1e-14)
+
+
+@pytest.mark.parametrize("eps_max", [1e-3, 1e-2, 1e-1])
+def test_asymmetric_vulnerability_bound(eps_max):
+    """Prop. 4.2.  Its proof bounds |Delta_a| by 2 eps_max (1 - p_a(z_c)) at a
+    point z_c of the segment; log p_a is concave along the segment, so the
+    smallest p_a(z_c) sits at an end point and the testable form is
+    |Delta_a| <= 2 eps_max (1 - min(p_a, p'_a))."""
+    rng = np.random.default_rng(17)
+    T, V = 64, 300
+    z = _rows(rng, T, V, scale=3.0)
+    zi = z + rng.uniform(-eps_max, eps_max, size=z.shape)
+    for pick in ("argmax", "random"):
+        ids = z.argmax(1) if pick == "argmax" else rng.integers(0, V, size=T)
+        tr = oracle.dvp_rows_f64(z, ids, 0.0).train
+        inf = oracle.dvp_rows_f64(zi, ids, 0.0).train
+        delta = tr.logp - inf.logp
+        p_min = np.minimum(np.exp(tr.logp), np.exp(inf.logp))
+        assert (np.abs(delta) <= 2 * eps_max * (1 - p_min) + 1e-12).all()
+        if pick == "argmax":
+            # the bound contracts for high-probability tokens
+            assert np.abs(delta).max() < 2 * eps_max
+
+
+def test_log_ratio_sign_and_conventions():
+    """Delta = train - infer (Thm. 4.1); ratio zero when a leaves the training
+    set (remark after Thm. 5.3); +inf when only the inference set drops it."""
+    z = np.array([[5.0, 4.0, 2.0, -1.0]] * 3, dtype=np.float32)
+    zi = z.copy()
+    zi[0, 1] = 4.5                      # token 1 more likely under infer
+    zi[1, 2] = -4.0                     # row 1: token 2 pruned on the infer side only
+    z[2, 2] = -4.0                      # row 2: token 2 pruned on the train side only
+    ids = np.array([1, 2, 2])
+    res = oracle.dvp_rows(z, ids, 0.02, infer=zi)          # ln(0.02) = -3.9: tau = 1.09
+    assert res.log_ratio[0] < 0 and np.isfinite(res.log_ratio[0])
+    assert res.log_ratio[0] == pytest.approx(res.train.logp_mp[0] - res.infer.logp_mp[0])
+    assert res.train.member.tolist() == [1, 1, 0] and res.infer.member.tolist() == [1, 0, 1]
+    assert res.log_ratio[1] == np.inf and res.log_ratio[2] == -np.inf
+
+
+def test_printed_constants():
+    with open(os.path.join(GOLDEN, "paper_constants.txt")) as f:
+        rows = [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 3
+    for name, expr, printed, digits, *_ in rows:
+        value = eval(expr, {"exp": math.exp})
+        assert float(f"{value:.{int(digits) - 1}e}") == float(printed), name
+    # the default threshold enters the oracle as log(rho) = -13
+    z = np.array([[0.0, -12.999, -13.001]])
+    res = oracle.dvp_rows_f64(z, np.array([0]), math.exp(-13), want_mask=True)
+    assert res.train.mask.tolist() == [[1, 1, 0]]
+
+
+def test_storage_types_widen_exactly_and_strides_are_honoured():
+    rng = np.random.default_rng(21)
+    x = torch.from_numpy(rng.normal(size=(5, 64)).astype(np.float32) * 4)
+    ids = rng.integers(0, 48, size=5)
+    for dt, code in ((torch.bfloat16, oracle.BF16), (torch.float16, oracle.F16)):
+        xs = x.to(dt)
+        bits = xs.view(torch.int16).numpy().view(np.uint16)
+        got = oracle.dvp_rows(bits[:, :48], ids, 1e-2, dtype=code)       # row stride 64 > V 48
+        want = oracle.dvp_rows_f64(xs[:, :48].to(torch.float64).numpy(), ids, 1e-2)
+        for name in ("max", "lse", "lse_safe", "logp_mp", "count"):
+            assert np.array_equal(getattr(got.train, name), getattr(want.train, name)), name
+    sub = torch.tensor([1e-7, -3e-6, 6e-5, 0.0], dtype=torch.float16)   # subnormal halves
+    got = oracle.dvp_rows(sub.view(torch.int16).numpy().view(np.uint16)[None, :], np.array([2]), 0.0,
+                          dtype=oracle.F16)
+    assert got.train.max[0] == float(sub.max())
+
+
+def test_batch_driver_threads_agree_and_no_id_rows():
+    rng = np.random.default_rng(23)
+    z = (rng.normal(size=(37, 130)) * 3).astype(np.float32)
+    zi = (z + rng.normal(size=z.shape) * 0.01).astype(np.float32)
+    ids = rng.integers(0, 130, size=37)
+    ids[5] = -1
+    g = rng.normal(size=37)
+    r1 = oracle.dvp_rows(z, ids, 1e-3, infer=zi, upstream=g, want_grad=True, want_mask=True, threads=1)
+    r4 = oracle.dvp_rows(z, ids, 1e-3, infer=zi, upstream=g, want_grad=True, want_mask=True, threads=4)
+    assert r4.threads == 4
+    assert np.array_equal(r1.grad, r4.grad) and np.array_equal(r1.train.mask, r4.train.mask)
+    np.testing.assert_array_equal(r1.log_ratio, r4.log_ratio)
+    assert np.isnan(r1.train.logp_mp[5]) and (r1.grad[5] == 0).all() and r1.train.count[5] >= 1
+
+
+def test_fused_lmhead_matches_autograd_through_the_head():
+    """Chain rule of Prop. 5.6 part 2 through z = h W^T, by torch autograd."""
+    rng = np.random.default_rng(29)
+    T, H, V, rho = 5, 8, 23, 5e-2
+    hb = torch.from_numpy(rng.normal(size=(T, H)).astype(np.float32)).to(torch.bfloat16)
+    wb = torch.from_numpy((rng.normal(size=(V, H)) * 0.5).astype(np.float32)).to(torch.bfloat16)
+    h = hb.to(torch.float64).requires_grad_(True)
+    w = wb.to(torch.float64).requires_grad_(True)
+    z = h @ w.t()
+    zi = (z.detach() + torch.from_numpy(rng.normal(size=(T, V)) * 0.02)).to(torch.bfloat16)
+    ids = rng.integers(0, V, size=T)
+    ids[:3] = z.detach().numpy().argmax(1)[:3]
+    g = torch.from_numpy(rng.normal(size=T))
+    with torch.no_grad():
+        pruned = z < z.max(dim=-1, keepdim=True).values + math.log(rho)
+    logp = torch.log_softmax(torch.where(pruned, torch.tensor(-math.inf, dtype=z.dtype), z), dim=-1)
+    logp = logp[torch.arange(T), torch.from_numpy(ids)]
+    member = torch.isfinite(logp)
+    (logp[member] * g[member]).sum().backward()
+    bits = lambda x: x.view(torch.int16).numpy().view(np.uint16)
+    res = oracle.dvp_fused_lmhead(bits(hb), bits(wb), bits(zi), ids, rho, g.numpy())
+    np.testing.assert_allclose(res.logits, z.detach().numpy(), atol=1e-13)
+    np.testing.assert_allclose(res.d_hidden, h.grad.numpy(), atol=1e-12)
+    np.testing.assert_allclose(res.d_w, w.grad.numpy(), atol=1e-12)
+    want = logp.detach().numpy()
+    np.testing.assert_allclose(res.rows.train.logp_mp[member.numpy()], want[member.numpy()], atol=1e-12)
+    # infer side: an ordinary row pass on the stored bf16 logits
+    ref_i = oracle.dvp_rows(bits(zi), ids, rho, dtype=oracle.BF16)
+    assert np.array_equal(res.rows.infer.logp_mp, ref_i.train.logp_mp)
