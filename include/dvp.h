@@ -1,0 +1,238 @@
+/*
+ * dvp.h -- C ABI of the B200 (sm_100a) Dynamic Vocabulary Pruning library.
+ *
+ * The library turns [T, V] logit matrices into the pruned objective of
+ * "Dynamic Vocabulary Pruning: Stable LLM-RL by Taming the Tail"
+ * (arXiv 2512.23087).  Per token row (one state s), with logits z, sampled
+ * token a, threshold rho and L = ln(rho):
+ *
+ *   safe set      V_S = { k : z_k >= max_j z_j + L }        Def. 5.1, in the
+ *                 logit-space form of App. A (protocol 2); equality is kept
+ *   coverage      Z = sum_{k in V_S} pi(k)                   Def. 5.2
+ *   pruned policy pi^mp(a) = pi(a) / Z on V_S, 0 elsewhere   Def. 5.2, Prop. 5.6(1)
+ *   gradient      d log pi^mp(a) / d z_k = 1[k=a] - pi^mp(k) on V_S, 0 off it,
+ *                 safe set held fixed                        Prop. 5.4, Prop. 5.6(2)
+ *   log-ratio     ln pi^mp_train(a) - ln pi^mp_infer(a)      Thm. 4.1 (sign), Thm. 5.3,
+ *                                                            App. A (protocol 4)
+ *
+ * Conventions that hold for every entry point
+ *   - Every pointer marked "device" is a CUDA device pointer owned by the
+ *     caller; the library never allocates, frees or retains it.
+ *   - A call validates its arguments on the host, enqueues kernels on
+ *     `stream` (a cudaStream_t passed as void*) and returns without
+ *     synchronising.  Outputs are valid once the stream reaches that point.
+ *   - Return value: a dvp_status.  Host-detectable problems are reported
+ *     before anything is launched.  Problems only the device can see (a
+ *     sampled id outside [0, V)) set DVP_FLAG_BAD_ID for that token, give it
+ *     NaN log-probabilities and a zero gradient row; nothing traps.
+ *   - Matrices are row-major with a row stride `ld*` counted in elements.
+ *   - `struct_size` must equal sizeof of the struct the caller compiled with.
+ *   - Logits must be finite.  Behaviour on NaN or infinite logits is
+ *     unspecified (no fault, but the numbers mean nothing).
+ *   - rho lies in [0, 1].  rho = 0 keeps every token (full log-softmax);
+ *     rho = 1 keeps the argmax and its exact ties.
+ *   - The membership test is exact: it equals the comparison of the stored
+ *     logit, widened to double, against (double)max + log(rho) in double.
+ */
+#ifndef DVP_H_
+#define DVP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DVP_OK = 0,
+  DVP_ERR_INVALID_ARG = 1, /* null pointer, bad size, rho outside [0,1], ... */
+  DVP_ERR_UNSUPPORTED = 2, /* dtype, device architecture or size not handled */
+  DVP_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small     */
+  DVP_ERR_CUDA = 4         /* a CUDA runtime call failed                     */
+} dvp_status;
+
+typedef enum { DVP_F32 = 0, DVP_BF16 = 1, DVP_F16 = 2 } dvp_dtype;
+typedef enum { DVP_ID_I64 = 0, DVP_ID_I32 = 1 } dvp_id_dtype;
+
+/* bits of the per-token flags byte */
+enum {
+  DVP_FLAG_IN_TRAIN = 1, /* a is in the training safe set V_S               */
+  DVP_FLAG_IN_INFER = 2, /* a is in the inference safe set V'_S             */
+  DVP_FLAG_NO_ID = 64,   /* id < 0: row statistics only                     */
+  DVP_FLAG_BAD_ID = 128  /* id >= V                                         */
+};
+
+enum { DVP_ENTRY_FORWARD = 0, DVP_ENTRY_BACKWARD = 1, DVP_ENTRY_FUSED_LMHEAD = 2 };
+
+/*
+ * Per-token outputs of one policy ("side"): each pointer is a device array of
+ * T elements and may be NULL when the caller does not want it.
+ */
+typedef struct {
+  float *max;       /* m = max_k z_k                                          */
+  float *lse;       /* ln sum_k e^{z_k}                  (full vocabulary)    */
+  float *lse_safe;  /* ln sum_{k in V_S} e^{z_k}                              */
+  float *logp;      /* ln pi(a)                                               */
+  float *logp_mp;   /* ln pi^mp(a); -inf when a is pruned      (Def. 5.2)     */
+  float *comp_mp;   /* 1 - pi^mp(a), summed without the a term (no cancellation) */
+  int32_t *count;   /* |V_S|                                                  */
+  uint32_t *mask;   /* [T, ceil(V/32)] packed: bit (k%32) of word k/32 set    */
+                    /* when k in V_S; padding bits of the last word are zero  */
+} dvp_side_out;
+
+/*
+ * dvp_forward -- Def. 5.1, Def. 5.2, Prop. 5.6(1) for the training and the
+ * inference logits, the per-token log-ratio of Thm. 5.3 / App. A protocol 4,
+ * and, when `upstream` and `grad_train` are both given, the gradient of
+ * Prop. 5.4 / Prop. 5.6(2) written in the same sweep over the training row.
+ *
+ *   train_logits  device [T, ld_train], required
+ *   infer_logits  device [T, ld_infer] or NULL (then `infer`, `log_ratio`
+ *                 must be NULL); same dtype as the training logits
+ *   ids           device [T] int64 or int32; id < 0: statistics only
+ *   upstream      device [T] float32: g_t = dLoss / d ln pi^mp_train(a_t)
+ *   grad_train    device [T, ld_grad] of grad_dtype: g_t (1[k=a] - pi^mp(k))
+ *                 on V_S, 0 off it, the whole row 0 when a is not in V_S;
+ *                 rounded to nearest-even in grad_dtype
+ *   log_ratio     device [T] float32: ln pi^mp_train(a) - ln pi^mp_infer(a);
+ *                 -inf when a is outside V_S (importance ratio zero, remark
+ *                 after Thm. 5.3), +inf when a is in V_S but outside V'_S
+ *   flags         device [T] bytes, DVP_FLAG_* bits
+ *   launch_hint   0 = library default; otherwise threads per block in the low
+ *                 16 bits and loads in flight per thread in the next 8 bits
+ *                 (tuning only, results do not depend on it)
+ *
+ * Rows whose start is 16-byte aligned in all three matrices take the
+ * vectorised kernels; any other layout takes a scalar kernel, same results.
+ * Needs no workspace.  Errors: DVP_ERR_INVALID_ARG for NULL required
+ * pointers, T < 0, V < 1, ld < V, rho outside [0,1] or NaN, upstream without
+ * grad_train or the reverse; DVP_ERR_UNSUPPORTED for unknown dtypes or a row
+ * too long for the on-chip row summary (V above about 1.7 million elements).
+ * T = 0 is a valid no-op.
+ */
+typedef struct {
+  uint32_t struct_size;
+  int32_t logits_dtype; /* dvp_dtype of train_logits and infer_logits */
+  int32_t grad_dtype;   /* dvp_dtype of grad_train                    */
+  int32_t id_dtype;     /* dvp_id_dtype                               */
+  int64_t T, V;
+  int64_t ld_train, ld_infer, ld_grad;
+  double rho;
+  const void *train_logits;
+  const void *infer_logits;
+  const void *ids;
+  const float *upstream;
+  void *grad_train;
+  dvp_side_out train;
+  dvp_side_out infer;
+  float *log_ratio;
+  uint8_t *flags;
+  void *stream;
+  uint32_t launch_hint;
+  uint32_t reserved_;
+} dvp_forward_args;
+
+int dvp_forward(const dvp_forward_args *args);
+
+/*
+ * dvp_backward -- Prop. 5.4 / Prop. 5.6(2) as a stand-alone streaming map for
+ * callers whose upstream gradient depends on the forward outputs.  Takes the
+ * vectors a previous dvp_forward saved for the same logits, ids and rho:
+ *
+ *   max_t, lse_safe_t, flags   device [T], required (from dvp_forward)
+ *   comp_mp_t                  device [T] or NULL; when NULL the a-th entry is
+ *                              g (1 - exp(z_a - lse_safe)), which loses digits
+ *                              as pi^mp(a) -> 1
+ * Reads the training logits once and writes grad_train once.  Same error
+ * rules as dvp_forward.  Needs no workspace.
+ */
+typedef struct {
+  uint32_t struct_size;
+  int32_t logits_dtype, grad_dtype, id_dtype;
+  int64_t T, V;
+  int64_t ld_train, ld_grad;
+  double rho;
+  const void *train_logits;
+  const void *ids;
+  const float *upstream;
+  const float *max_t;
+  const float *lse_safe_t;
+  const float *comp_mp_t;
+  const uint8_t *flags;
+  void *grad_train;
+  void *stream;
+  uint32_t launch_hint;
+  uint32_t reserved_;
+} dvp_backward_args;
+
+int dvp_backward(const dvp_backward_args *args);
+
+/*
+ * dvp_fused_lmhead_forward_backward -- the same objective with the training
+ * logits produced on the fly as z = hidden x W_vocab^T (bf16 operands, fp32
+ * accumulation on the tensor cores), so the [T, V] training logits are never
+ * stored: rows are processed in panels of `panel_rows` tokens whose logits
+ * live in the workspace only.  The gradient flows through the linear head by
+ * the chain rule of Prop. 5.6(2): d_hidden = G W and d_w = G^T hidden with
+ * G = dLoss/dz as in dvp_forward.
+ *
+ *   hidden        device [T, ld_hidden] bf16
+ *   w_vocab       device [V, ld_w] bf16
+ *   infer_logits  device [T, ld_infer] bf16 (what the inference engine
+ *                 computed for the same parameters), or NULL
+ *   d_hidden      device [T, ld_dh] float32, overwritten
+ *   d_w           device [V, ld_dw] float32; overwritten, or added to when
+ *                 accumulate_dw != 0
+ *   workspace     device, 256-byte aligned, at least
+ *                 dvp_workspace_bytes(DVP_ENTRY_FUSED_LMHEAD, args) bytes
+ *   panel_rows    0 = library default; otherwise a multiple of 128
+ *
+ * H must be a multiple of 64 and rows of hidden, w_vocab must start on
+ * 16-byte boundaries (DVP_ERR_UNSUPPORTED otherwise).  Membership is decided
+ * on the fp32-accumulated logits, so a token whose logit sits within rounding
+ * distance of the threshold may fall on either side.
+ */
+typedef struct {
+  uint32_t struct_size;
+  int32_t id_dtype;
+  int64_t T, H, V;
+  int64_t ld_hidden, ld_w, ld_infer, ld_dh, ld_dw;
+  double rho;
+  const void *hidden;
+  const void *w_vocab;
+  const void *infer_logits;
+  const void *ids;
+  const float *upstream;
+  float *d_hidden;
+  float *d_w;
+  int32_t accumulate_dw;
+  int32_t panel_rows;
+  dvp_side_out train;
+  dvp_side_out infer;
+  float *log_ratio;
+  uint8_t *flags;
+  void *workspace;
+  size_t workspace_bytes;
+  void *stream;
+} dvp_fused_args;
+
+int dvp_fused_lmhead_forward_backward(const dvp_fused_args *args);
+
+/*
+ * Bytes of device workspace the entry point needs for `args` (a pointer to
+ * that entry point's args struct; only sizes and dtypes are read).  Returns 0
+ * for entry points that need none and for invalid arguments.
+ */
+size_t dvp_workspace_bytes(int entry_point, const void *args);
+
+/* Static, human-readable name of a dvp_status value. */
+const char *dvp_status_string(int status);
+
+/* Library version, major * 10000 + minor * 100 + patch. */
+int dvp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DVP_H_ */

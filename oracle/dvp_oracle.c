@@ -179,6 +179,7 @@ void dvp_oracle_side_grad(const double *z, int64_t V, int64_t a, double g,
  * training set but outside the inference set: r = +inf.
  */
 double dvp_oracle_log_ratio(const oracle_side *tr, const oracle_side *inf) {
+  if (isnan(tr->logp)) return NAN; /* no sampled token in this row */
   if (!tr->member) return -INFINITY;
   if (!inf->member) return INFINITY;
   return tr->logp_mp - inf->logp_mp;

@@ -1,0 +1,342 @@
+"""ctypes binding of the C ABI in ``include/dvp.h``.
+
+Argument marshalling only: tensors are turned into raw device pointers and
+sizes, outputs are allocated with torch, and every step of the computation
+runs in the CUDA library.  There is no fallback: if ``libdvp_b200.so`` has not
+been built, the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from types import SimpleNamespace
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdvp_b200.so")
+
+DVP_OK, DVP_ERR_INVALID_ARG, DVP_ERR_UNSUPPORTED, DVP_ERR_WORKSPACE, DVP_ERR_CUDA = range(5)
+DVP_F32, DVP_BF16, DVP_F16 = 0, 1, 2
+DVP_ID_I64, DVP_ID_I32 = 0, 1
+DVP_FLAG_IN_TRAIN, DVP_FLAG_IN_INFER, DVP_FLAG_NO_ID, DVP_FLAG_BAD_ID = 1, 2, 64, 128
+DVP_ENTRY_FORWARD, DVP_ENTRY_BACKWARD, DVP_ENTRY_FUSED_LMHEAD = 0, 1, 2
+
+EXPORTS = ("dvp_forward", "dvp_backward", "dvp_fused_lmhead_forward_backward",
+           "dvp_workspace_bytes", "dvp_status_string", "dvp_version")
+
+_DTYPES = {torch.float32: DVP_F32, torch.bfloat16: DVP_BF16, torch.float16: DVP_F16}
+_SIDE_FIELDS = ("max", "lse", "lse_safe", "logp", "logp_mp", "comp_mp", "count", "mask")
+
+
+class DvpError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+class SideOut(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in _SIDE_FIELDS]
+
+
+class ForwardArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("logits_dtype", ctypes.c_int32),
+        ("grad_dtype", ctypes.c_int32),
+        ("id_dtype", ctypes.c_int32),
+        ("T", ctypes.c_int64),
+        ("V", ctypes.c_int64),
+        ("ld_train", ctypes.c_int64),
+        ("ld_infer", ctypes.c_int64),
+        ("ld_grad", ctypes.c_int64),
+        ("rho", ctypes.c_double),
+        ("train_logits", ctypes.c_void_p),
+        ("infer_logits", ctypes.c_void_p),
+        ("ids", ctypes.c_void_p),
+        ("upstream", ctypes.c_void_p),
+        ("grad_train", ctypes.c_void_p),
+        ("train", SideOut),
+        ("infer", SideOut),
+        ("log_ratio", ctypes.c_void_p),
+        ("flags", ctypes.c_void_p),
+        ("stream", ctypes.c_void_p),
+        ("launch_hint", ctypes.c_uint32),
+        ("reserved_", ctypes.c_uint32),
+    ]
+
+
+class BackwardArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("logits_dtype", ctypes.c_int32),
+        ("grad_dtype", ctypes.c_int32),
+        ("id_dtype", ctypes.c_int32),
+        ("T", ctypes.c_int64),
+        ("V", ctypes.c_int64),
+        ("ld_train", ctypes.c_int64),
+        ("ld_grad", ctypes.c_int64),
+        ("rho", ctypes.c_double),
+        ("train_logits", ctypes.c_void_p),
+        ("ids", ctypes.c_void_p),
+        ("upstream", ctypes.c_void_p),
+        ("max_t", ctypes.c_void_p),
+        ("lse_safe_t", ctypes.c_void_p),
+        ("comp_mp_t", ctypes.c_void_p),
+        ("flags", ctypes.c_void_p),
+        ("grad_train", ctypes.c_void_p),
+        ("stream", ctypes.c_void_p),
+        ("launch_hint", ctypes.c_uint32),
+        ("reserved_", ctypes.c_uint32),
+    ]
+
+
+class FusedArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("id_dtype", ctypes.c_int32),
+        ("T", ctypes.c_int64),
+        ("H", ctypes.c_int64),
+        ("V", ctypes.c_int64),
+        ("ld_hidden", ctypes.c_int64),
+        ("ld_w", ctypes.c_int64),
+        ("ld_infer", ctypes.c_int64),
+        ("ld_dh", ctypes.c_int64),
+        ("ld_dw", ctypes.c_int64),
+        ("rho", ctypes.c_double),
+        ("hidden", ctypes.c_void_p),
+        ("w_vocab", ctypes.c_void_p),
+        ("infer_logits", ctypes.c_void_p),
+        ("ids", ctypes.c_void_p),
+        ("upstream", ctypes.c_void_p),
+        ("d_hidden", ctypes.c_void_p),
+        ("d_w", ctypes.c_void_p),
+        ("accumulate_dw", ctypes.c_int32),
+        ("panel_rows", ctypes.c_int32),
+        ("train", SideOut),
+        ("infer", SideOut),
+        ("log_ratio", ctypes.c_void_p),
+        ("flags", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_size_t),
+        ("stream", ctypes.c_void_p),
+    ]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load ``libdvp_b200.so``; raises if it is missing (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2512_23087_b200.build`; "
+                "this package has no CPU or PyTorch fallback")
+        lib = ctypes.CDLL(LIB_PATH)
+        lib.dvp_forward.argtypes = [ctypes.POINTER(ForwardArgs)]
+        lib.dvp_forward.restype = ctypes.c_int
+        lib.dvp_backward.argtypes = [ctypes.POINTER(BackwardArgs)]
+        lib.dvp_backward.restype = ctypes.c_int
+        lib.dvp_fused_lmhead_forward_backward.argtypes = [ctypes.POINTER(FusedArgs)]
+        lib.dvp_fused_lmhead_forward_backward.restype = ctypes.c_int
+        lib.dvp_workspace_bytes.argtypes = [ctypes.c_int, ctypes.c_void_p]
+        lib.dvp_workspace_bytes.restype = ctypes.c_size_t
+        lib.dvp_status_string.argtypes = [ctypes.c_int]
+        lib.dvp_status_string.restype = ctypes.c_char_p
+        lib.dvp_version.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load_library().dvp_status_string(int(status)).decode()
+
+
+def _ptr(t: torch.Tensor | None):
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+def _check_matrix(name: str, x: torch.Tensor):
+    if x.dim() != 2 or x.stride(1) != 1:
+        raise ValueError(f"{name} must be 2-D with unit inner stride")
+    if not x.is_cuda:
+        raise ValueError(f"{name} must live on a CUDA device")
+
+
+def _side(device, T: int, V: int, want_mask: bool):
+    o = SimpleNamespace()
+    for n in ("max", "lse", "lse_safe", "logp", "logp_mp", "comp_mp"):
+        setattr(o, n, torch.empty(T, dtype=torch.float32, device=device))
+    o.count = torch.empty(T, dtype=torch.int32, device=device)
+    o.mask = torch.empty(T, (V + 31) // 32, dtype=torch.int32, device=device) if want_mask else None
+    s = SideOut(*(_ptr(getattr(o, n)) for n in _SIDE_FIELDS))
+    return o, s
+
+
+def _id_dtype(ids: torch.Tensor) -> int:
+    if ids.dtype == torch.int64:
+        return DVP_ID_I64
+    if ids.dtype == torch.int32:
+        return DVP_ID_I32
+    raise TypeError("ids must be int64 or int32")
+
+
+def dvp_forward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, *,
+                infer_logits: torch.Tensor | None = None, upstream: torch.Tensor | None = None,
+                grad_train: torch.Tensor | None = None, grad_dtype: torch.dtype | None = None,
+                want_mask: bool = False, stream=None, launch_hint: int = 0, out=None):
+    """Pruned log-probabilities of the sampled tokens for the training and the
+    inference logits (Def. 5.1, Def. 5.2), their log-ratio, and, when
+    ``upstream`` is given, dLoss/dlogits (Prop. 5.4) in the same launch.
+
+    Returns a namespace with ``train`` / ``infer`` (per-token tensors),
+    ``log_ratio``, ``flags`` and ``grad_train``.  Pass the namespace of an
+    earlier call as ``out`` to reuse its buffers.
+    """
+    lib = load_library()
+    _check_matrix("train_logits", train_logits)
+    T, V = train_logits.shape
+    dev = train_logits.device
+    a = ForwardArgs()
+    a.struct_size = ctypes.sizeof(ForwardArgs)
+    a.logits_dtype = _DTYPES[train_logits.dtype]
+    a.id_dtype = _id_dtype(ids)
+    a.T, a.V, a.rho = T, V, float(rho)
+    a.ld_train = train_logits.stride(0)
+    a.train_logits = _ptr(train_logits)
+    a.ids = _ptr(ids)
+    res = out if out is not None else SimpleNamespace(train=None, infer=None, log_ratio=None,
+                                                      flags=None, grad_train=None)
+    if out is None:
+        res.train, res._train_struct = _side(dev, T, V, want_mask)
+        res.flags = torch.empty(T, dtype=torch.uint8, device=dev)
+    a.train = res._train_struct
+    a.flags = _ptr(res.flags)
+    if infer_logits is not None:
+        _check_matrix("infer_logits", infer_logits)
+        if infer_logits.dtype != train_logits.dtype or infer_logits.shape != train_logits.shape:
+            raise ValueError("infer_logits must match train_logits in dtype and shape")
+        a.infer_logits = _ptr(infer_logits)
+        a.ld_infer = infer_logits.stride(0)
+        if out is None:
+            res.infer, res._infer_struct = _side(dev, T, V, want_mask)
+            res.log_ratio = torch.empty(T, dtype=torch.float32, device=dev)
+        a.infer = res._infer_struct
+        a.log_ratio = _ptr(res.log_ratio)
+    if upstream is not None:
+        if upstream.dtype != torch.float32:
+            raise TypeError("upstream must be float32")
+        if grad_train is None:
+            grad_train = res.grad_train
+        if grad_train is None:
+            grad_train = torch.empty(T, V, dtype=grad_dtype or train_logits.dtype, device=dev)
+        _check_matrix("grad_train", grad_train)
+        res.grad_train = grad_train
+        a.upstream = _ptr(upstream)
+        a.grad_train = _ptr(grad_train)
+        a.grad_dtype = _DTYPES[grad_train.dtype]
+        a.ld_grad = grad_train.stride(0)
+    a.stream = _stream(stream)
+    a.launch_hint = launch_hint
+    st = lib.dvp_forward(ctypes.byref(a))
+    if st != DVP_OK:
+        raise DvpError(st, "dvp_forward")
+    return res
+
+
+def dvp_backward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, upstream: torch.Tensor,
+                 saved, *, grad_train: torch.Tensor | None = None,
+                 grad_dtype: torch.dtype | None = None, use_comp: bool = True, stream=None,
+                 launch_hint: int = 0) -> torch.Tensor:
+    """dLoss/dlogits from the vectors an earlier ``dvp_forward`` saved
+    (``saved`` = its result namespace) and a per-token upstream gradient."""
+    lib = load_library()
+    _check_matrix("train_logits", train_logits)
+    T, V = train_logits.shape
+    if grad_train is None:
+        grad_train = torch.empty(T, V, dtype=grad_dtype or train_logits.dtype,
+                                 device=train_logits.device)
+    _check_matrix("grad_train", grad_train)
+    a = BackwardArgs()
+    a.struct_size = ctypes.sizeof(BackwardArgs)
+    a.logits_dtype = _DTYPES[train_logits.dtype]
+    a.grad_dtype = _DTYPES[grad_train.dtype]
+    a.id_dtype = _id_dtype(ids)
+    a.T, a.V, a.rho = T, V, float(rho)
+    a.ld_train, a.ld_grad = train_logits.stride(0), grad_train.stride(0)
+    a.train_logits, a.ids, a.upstream = _ptr(train_logits), _ptr(ids), _ptr(upstream)
+    a.max_t, a.lse_safe_t = _ptr(saved.train.max), _ptr(saved.train.lse_safe)
+    a.comp_mp_t = _ptr(saved.train.comp_mp) if use_comp else None
+    a.flags = _ptr(saved.flags)
+    a.grad_train = _ptr(grad_train)
+    a.stream = _stream(stream)
+    a.launch_hint = launch_hint
+    st = lib.dvp_backward(ctypes.byref(a))
+    if st != DVP_OK:
+        raise DvpError(st, "dvp_backward")
+    return grad_train
+
+
+def dvp_workspace_bytes(entry_point: int, args: ctypes.Structure) -> int:
+    return int(load_library().dvp_workspace_bytes(int(entry_point), ctypes.byref(args)))
+
+
+def dvp_fused_lmhead_forward_backward(hidden: torch.Tensor, w_vocab: torch.Tensor, ids: torch.Tensor,
+                                      rho: float, upstream: torch.Tensor, *,
+                                      infer_logits: torch.Tensor | None = None,
+                                      d_w: torch.Tensor | None = None, accumulate_dw: bool = False,
+                                      panel_rows: int = 0, workspace: torch.Tensor | None = None,
+                                      stream=None):
+    """Pruned log-probabilities and gradients with respect to ``hidden`` and
+    ``w_vocab`` with the training logits hidden x w_vocab^T produced panel by
+    panel inside the library and never stored as a [T, V] matrix."""
+    lib = load_library()
+    _check_matrix("hidden", hidden)
+    _check_matrix("w_vocab", w_vocab)
+    T, H = hidden.shape
+    V = w_vocab.shape[0]
+    dev = hidden.device
+    if hidden.dtype != torch.bfloat16 or w_vocab.dtype != torch.bfloat16:
+        raise TypeError("hidden and w_vocab must be bfloat16")
+    a = FusedArgs()
+    a.struct_size = ctypes.sizeof(FusedArgs)
+    a.id_dtype = _id_dtype(ids)
+    a.T, a.H, a.V, a.rho = T, H, V, float(rho)
+    a.ld_hidden, a.ld_w = hidden.stride(0), w_vocab.stride(0)
+    a.hidden, a.w_vocab, a.ids, a.upstream = _ptr(hidden), _ptr(w_vocab), _ptr(ids), _ptr(upstream)
+    res = SimpleNamespace(infer=None, log_ratio=None)
+    res.train, a.train = _side(dev, T, V, False)
+    res.flags = torch.empty(T, dtype=torch.uint8, device=dev)
+    a.flags = _ptr(res.flags)
+    if infer_logits is not None:
+        _check_matrix("infer_logits", infer_logits)
+        if infer_logits.dtype != torch.bfloat16:
+            raise TypeError("infer_logits must be bfloat16")
+        a.infer_logits, a.ld_infer = _ptr(infer_logits), infer_logits.stride(0)
+        res.infer, a.infer = _side(dev, T, V, False)
+        res.log_ratio = torch.empty(T, dtype=torch.float32, device=dev)
+        a.log_ratio = _ptr(res.log_ratio)
+    res.d_hidden = torch.empty(T, H, dtype=torch.float32, device=dev)
+    res.d_w = d_w if d_w is not None else torch.empty(V, H, dtype=torch.float32, device=dev)
+    a.d_hidden, a.ld_dh = _ptr(res.d_hidden), res.d_hidden.stride(0)
+    a.d_w, a.ld_dw = _ptr(res.d_w), res.d_w.stride(0)
+    a.accumulate_dw = int(accumulate_dw)
+    a.panel_rows = int(panel_rows)
+    need = dvp_workspace_bytes(DVP_ENTRY_FUSED_LMHEAD, a)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    res.workspace = workspace
+    a.workspace, a.workspace_bytes = _ptr(workspace), workspace.numel() * workspace.element_size()
+    a.stream = _stream(stream)
+    st = lib.dvp_fused_lmhead_forward_backward(ctypes.byref(a))
+    if st != DVP_OK:
+        raise DvpError(st, "dvp_fused_lmhead_forward_backward")
+    return res

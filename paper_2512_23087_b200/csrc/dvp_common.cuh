@@ -1,0 +1,299 @@
+// Shared device helpers of the DVP row kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dvp.h"
+
+namespace dvp {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kNegInf = -__builtin_huge_valf();
+
+// e^{x} for x already multiplied by log2(e): one MUFU op, flushes denormals.
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// 16-byte read-only load that does not allocate in L1: each logit is consumed
+// once per sweep, re-reads are served by L2.
+__device__ __forceinline__ uint4 ld_stream16(const void *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+// Streaming stores (evict-first): the gradient is written once and not read
+// again by this library.
+__device__ __forceinline__ void st_stream16(void *p, uint4 v) {
+  asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
+               "r"(v.w)
+               : "memory");
+}
+__device__ __forceinline__ void st_stream8(void *p, uint2 v) {
+  asm volatile("st.global.cs.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(v.x), "r"(v.y) : "memory");
+}
+
+// ---- storage types ---------------------------------------------------------
+
+template <typename T>
+struct Storage;
+
+template <>
+struct Storage<float> {
+  static constexpr int kPerVec = 4;  // elements in 16 bytes
+  static __device__ __forceinline__ void unpack(uint4 r, float *x) {
+    x[0] = __uint_as_float(r.x);
+    x[1] = __uint_as_float(r.y);
+    x[2] = __uint_as_float(r.z);
+    x[3] = __uint_as_float(r.w);
+  }
+  static __device__ __forceinline__ float widen(float v) { return v; }
+  static __device__ __forceinline__ float narrow(float v) { return v; }
+};
+
+template <>
+struct Storage<__nv_bfloat16> {
+  static constexpr int kPerVec = 8;
+  static __device__ __forceinline__ void unpack(uint4 r, float *x) {
+    // a bfloat16 is the upper half of a binary32
+    x[0] = __uint_as_float(r.x << 16);
+    x[1] = __uint_as_float(r.x & 0xffff0000u);
+    x[2] = __uint_as_float(r.y << 16);
+    x[3] = __uint_as_float(r.y & 0xffff0000u);
+    x[4] = __uint_as_float(r.z << 16);
+    x[5] = __uint_as_float(r.z & 0xffff0000u);
+    x[6] = __uint_as_float(r.w << 16);
+    x[7] = __uint_as_float(r.w & 0xffff0000u);
+  }
+  static __device__ __forceinline__ float widen(__nv_bfloat16 v) { return __bfloat162float(v); }
+  static __device__ __forceinline__ __nv_bfloat16 narrow(float v) { return __float2bfloat16_rn(v); }
+};
+
+template <>
+struct Storage<__half> {
+  static constexpr int kPerVec = 8;
+  static __device__ __forceinline__ void unpack(uint4 r, float *x) {
+    const __half2 *h = reinterpret_cast<const __half2 *>(&r);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float2 f = __half22float2(h[i]);
+      x[2 * i] = f.x;
+      x[2 * i + 1] = f.y;
+    }
+  }
+  static __device__ __forceinline__ float widen(__half v) { return __half2float(v); }
+  static __device__ __forceinline__ __half narrow(float v) { return __float2half_rn(v); }
+};
+
+// Store N consecutive gradients (N = 4 or 8), round-to-nearest-even, to an
+// address aligned to N * sizeof(TG).
+template <typename TG, int N>
+__device__ __forceinline__ void store_grads(TG *dst, const float *g) {
+  if constexpr (sizeof(TG) == 4) {
+#pragma unroll
+    for (int i = 0; i < N; i += 4)
+      st_stream16(dst + i, make_uint4(__float_as_uint(g[i]), __float_as_uint(g[i + 1]),
+                                      __float_as_uint(g[i + 2]), __float_as_uint(g[i + 3])));
+  } else {
+    uint32_t w[N / 2];
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) {
+      TG lo = Storage<TG>::narrow(g[2 * i]), hi = Storage<TG>::narrow(g[2 * i + 1]);
+      w[i] = (uint32_t) * reinterpret_cast<uint16_t *>(&lo) |
+             ((uint32_t) * reinterpret_cast<uint16_t *>(&hi) << 16);
+    }
+    if constexpr (N == 8)
+      st_stream16(dst, make_uint4(w[0], w[1], w[2], w[3]));
+    else
+      st_stream8(dst, make_uint2(w[0], w[1]));
+  }
+}
+
+template <typename TG, int N>
+__device__ __forceinline__ void store_zeros(TG *dst) {
+  if constexpr (sizeof(TG) == 4) {
+#pragma unroll
+    for (int i = 0; i < N; i += 4) st_stream16(dst + i, make_uint4(0, 0, 0, 0));
+  } else if constexpr (N == 8) {
+    st_stream16(dst, make_uint4(0, 0, 0, 0));
+  } else {
+    st_stream8(dst, make_uint2(0, 0));
+  }
+}
+
+// ---- block reductions in a fixed order (bit-identical from run to run) ------
+
+// Partial log-sum-exp state: sum of e^{z - m} over the elements seen so far.
+struct MaxSum {
+  float m, s;
+};
+
+__device__ __forceinline__ MaxSum combine(MaxSum a, MaxSum b) {
+  const float m = fmaxf(a.m, b.m);
+  MaxSum r;
+  r.m = m;
+  // a side that has seen nothing carries m = -inf and contributes nothing
+  const float sa = a.m > kNegInf ? a.s * ex2((a.m - m) * kLog2e) : 0.f;
+  const float sb = b.m > kNegInf ? b.s * ex2((b.m - m) * kLog2e) : 0.f;
+  r.s = sa + sb;
+  return r;
+}
+
+// scratch: 64 floats of shared memory.  Result valid in every thread.
+__device__ __forceinline__ MaxSum block_reduce_maxsum(MaxSum v, float *scratch) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    MaxSum other;
+    other.m = __shfl_xor_sync(0xffffffffu, v.m, o);
+    other.s = __shfl_xor_sync(0xffffffffu, v.s, o);
+    // keep operand order independent of the lane so both partners agree
+    v = (lane & o) ? combine(other, v) : combine(v, other);
+  }
+  __syncthreads();  // scratch may still be read from an earlier reduction
+  if (lane == 0) {
+    scratch[warp] = v.m;
+    scratch[32 + warp] = v.s;
+  }
+  __syncthreads();
+  MaxSum r;
+  r.m = lane < nwarp ? scratch[lane] : kNegInf;
+  r.s = lane < nwarp ? scratch[32 + lane] : 0.f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    MaxSum other;
+    other.m = __shfl_xor_sync(0xffffffffu, r.m, o);
+    other.s = __shfl_xor_sync(0xffffffffu, r.s, o);
+    r = (lane & o) ? combine(other, r) : combine(r, other);
+  }
+  return r;
+}
+
+struct SumCount {
+  float s;
+  int n;
+};
+
+__device__ __forceinline__ SumCount block_reduce_sumcount(SumCount v, float *scratch) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float os = __shfl_xor_sync(0xffffffffu, v.s, o);
+    const int on = __shfl_xor_sync(0xffffffffu, v.n, o);
+    v.s = (lane & o) ? os + v.s : v.s + os;
+    v.n += on;
+  }
+  __syncthreads();
+  if (lane == 0) {
+    scratch[warp] = v.s;
+    reinterpret_cast<int *>(scratch)[32 + warp] = v.n;
+  }
+  __syncthreads();
+  SumCount r;
+  r.s = lane < nwarp ? scratch[lane] : 0.f;
+  r.n = lane < nwarp ? reinterpret_cast<int *>(scratch)[32 + lane] : 0;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float os = __shfl_xor_sync(0xffffffffu, r.s, o);
+    const int on = __shfl_xor_sync(0xffffffffu, r.n, o);
+    r.s = (lane & o) ? os + r.s : r.s + os;
+    r.n += on;
+  }
+  return r;
+}
+
+// ---- per-row bookkeeping shared by all row kernels ---------------------------
+
+struct RowParams {
+  const void *train, *infer, *ids;
+  const float *upstream;
+  void *grad;
+  long long T, V, ld_train, ld_infer, ld_grad;
+  double log_rho;  // ln(rho); -inf for rho = 0
+  int id_is_i32;
+  dvp_side_out out_t, out_i;
+  float *log_ratio;
+  uint8_t *flags;
+};
+
+__device__ __forceinline__ long long load_id(const void *ids, int is_i32, long long t) {
+  return is_i32 ? (long long)reinterpret_cast<const int *>(ids)[t]
+                : reinterpret_cast<const long long *>(ids)[t];
+}
+
+// Threshold in the logits' own precision: the smallest float that is >= the
+// double m + ln(rho).  For stored values that are floats (or narrower),
+// "z >= tau_f" then decides exactly as the double comparison does.
+__device__ __forceinline__ float threshold_f32(float m, double log_rho) {
+  return __double2float_ru((double)m + log_rho);
+}
+
+// Everything one side of one row reduces to.
+struct SideStats {
+  float m;       // row max
+  float s;       // sum_k e^{z_k - m}
+  float s_x;     // sum over the safe set without the sampled token
+  float e_a;     // e^{z_a - m} when a is in the safe set, else 0
+  float z_a;     // logit of the sampled token (0 when there is none)
+  float tau;     // threshold_f32(m, log_rho)
+  int n;         // |V_S|
+  int member;    // a in V_S
+};
+
+// Writes the per-token outputs of one side; called by one thread.
+__device__ __forceinline__ float finish_side(const dvp_side_out &o, long long t, const SideStats &st,
+                                             bool has_id, bool bad_id) {
+  const float s_safe = st.s_x + st.e_a;
+  const float log_s = logf(st.s), log_ss = logf(s_safe);
+  const float nan = __int_as_float(0x7fc00000);
+  float logp = nan, logp_mp = nan, comp = nan;
+  if (has_id) {
+    logp = (st.z_a - st.m) - log_s;
+    logp_mp = st.member ? (st.z_a - st.m) - log_ss : kNegInf;
+    comp = st.member ? st.s_x / s_safe : 1.f;
+  }
+  if (bad_id) logp = logp_mp = comp = nan;
+  if (o.max) o.max[t] = st.m;
+  if (o.lse) o.lse[t] = st.m + log_s;
+  if (o.lse_safe) o.lse_safe[t] = st.m + log_ss;
+  if (o.logp) o.logp[t] = logp;
+  if (o.logp_mp) o.logp_mp[t] = logp_mp;
+  if (o.comp_mp) o.comp_mp[t] = comp;
+  if (o.count) o.count[t] = st.n;
+  return logp_mp;
+}
+
+// ln pi^mp_train(a) - ln pi^mp_infer(a) with the conventions for pruned tokens.
+__device__ __forceinline__ float log_ratio_of(bool in_train, bool in_infer, float lt, float li) {
+  if (!in_train) return kNegInf;
+  if (!in_infer) return -kNegInf;
+  return lt - li;
+}
+
+// Arguments of the stand-alone backward map.
+struct BackwardParams {
+  const void *train, *ids;
+  const float *upstream, *max_t, *lse_safe_t, *comp_mp_t;
+  const uint8_t *flags;
+  void *grad;
+  long long T, V, ld_train, ld_grad;
+  double log_rho;
+  int id_is_i32;
+};
+
+// Launchers (dvp_rows.cu).  `hint`: threads per block in the low 16 bits, loads
+// in flight per thread in the next 8 bits, 0 = default.
+cudaError_t launch_row_kernels(const RowParams &p, int logits_dtype, int grad_dtype, uint32_t hint,
+                               cudaStream_t s);
+cudaError_t launch_backward_kernel(const BackwardParams &p, int logits_dtype, int grad_dtype,
+                                   uint32_t hint, cudaStream_t s);
+
+}  // namespace dvp

@@ -1,0 +1,154 @@
+"""Comparison of the CUDA library's outputs with the fp64 oracle.
+
+Tolerances (stated once, used by every parity test):
+  * row max, safe-set size, membership flags, packed mask: bit-exact, except
+    rows that hold a logit within 1e-6 relative of the threshold, which are
+    counted and reported (the exact comparison scheme makes none expected);
+  * log-probabilities (logp, logp_mp, log_ratio): 1e-4 absolute, infinities
+    and NaNs must coincide;
+  * lse, lse_safe: 1e-4 absolute plus one float32 rounding of the value (they
+    are float32 outputs whose magnitude can reach the hundreds);
+  * gradients: per row, ||G - G_oracle||_2 <= (1e-3 + u) ||G_oracle||_2 with u
+    the unit roundoff of the gradient's storage type (0 for float32, 2^-9 for
+    bfloat16, 2^-12 for float16): round-to-nearest storage alone contributes
+    up to u.  Rows where both are zero pass.  In addition every element must
+    sit within (1e-3 + u) |G_oracle| + 1e-30 of the oracle's element.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+
+LOGP_TOL = 1e-4
+GRAD_TOL = 1e-3
+UNIT_ROUNDOFF = {torch.float32: 0.0, torch.bfloat16: 2.0 ** -9, torch.float16: 2.0 ** -12}
+ORACLE_DTYPE = {torch.float32: oracle.F32, torch.bfloat16: oracle.BF16, torch.float16: oracle.F16}
+
+
+def to_oracle_storage(x: torch.Tensor) -> np.ndarray:
+    """Host copy of stored logits in the form the oracle reads (same bits)."""
+    x = x.detach().cpu()
+    if x.dtype == torch.float32:
+        return x.numpy()
+    return x.view(torch.int16).numpy().view(np.uint16)
+
+
+def run_oracle(train, infer, ids, rho, upstream=None, want_mask=False, threads=8):
+    return oracle.dvp_rows(
+        to_oracle_storage(train), ids.detach().cpu().numpy().astype(np.int64), rho,
+        dtype=ORACLE_DTYPE[train.dtype],
+        infer=to_oracle_storage(infer) if infer is not None else None,
+        upstream=upstream.detach().cpu().numpy().astype(np.float64) if upstream is not None else None,
+        want_grad=upstream is not None, want_mask=want_mask, threads=threads)
+
+
+def near_threshold_rows(stored: torch.Tensor, side) -> np.ndarray:
+    """Rows that hold a logit within 1e-6 relative of the threshold."""
+    z = stored.detach().cpu().to(torch.float64).numpy()
+    tau = side.tau[:, None]
+    with np.errstate(invalid="ignore"):
+        close = np.abs(z - tau) <= 1e-6 * np.abs(tau)
+    return close.any(axis=1)
+
+
+def _same_special(got: np.ndarray, want: np.ndarray, name: str):
+    assert np.array_equal(np.isnan(got), np.isnan(want)), f"{name}: NaN pattern differs"
+    assert np.array_equal(np.isposinf(got), np.isposinf(want)), f"{name}: +inf pattern differs"
+    assert np.array_equal(np.isneginf(got), np.isneginf(want)), f"{name}: -inf pattern differs"
+
+
+def _close(got, want, tol, name, rows=None):
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    if rows is not None:
+        got, want = got[rows], want[rows]
+    _same_special(got, want, name)
+    fin = np.isfinite(want)
+    err = np.abs(got[fin] - want[fin])
+    bound = tol(want[fin]) if callable(tol) else tol
+    worst = float((err - bound).max()) if err.size else -1.0
+    assert worst <= 0, f"{name}: max error {err.max():.3e} beyond tolerance"
+    return float(err.max()) if err.size else 0.0
+
+
+def unpack_mask(mask: torch.Tensor, V: int) -> np.ndarray:
+    words = mask.detach().cpu().numpy().view(np.uint32)
+    bits = np.unpackbits(words.view(np.uint8), axis=1, bitorder="little")
+    assert not bits[:, V:].any(), "padding bits of the packed mask must be zero"
+    return bits[:, :V]
+
+
+def check_side(got, want, stored, V, label, report):
+    """got: namespace of device tensors; want: oracle.Side."""
+    near = near_threshold_rows(stored, want)
+    ok = ~near
+    report[f"{label}_near_threshold_rows"] = int(near.sum())
+    assert np.array_equal(got.max.cpu().numpy().astype(np.float64), want.max), f"{label}.max"
+    cnt = got.count.cpu().numpy().astype(np.int64)
+    assert np.array_equal(cnt[ok], want.count[ok]), f"{label}.count"
+    report[f"{label}_count_mismatch_near"] = int((cnt[near] != want.count[near]).sum())
+    lse_tol = lambda w: LOGP_TOL + 2.0 ** -23 * np.abs(w)
+    report[f"{label}_lse_err"] = _close(got.lse.cpu(), want.lse, lse_tol, f"{label}.lse")
+    report[f"{label}_lse_safe_err"] = _close(got.lse_safe.cpu(), want.lse_safe, lse_tol,
+                                             f"{label}.lse_safe", ok)
+    report[f"{label}_logp_err"] = _close(got.logp.cpu(), want.logp, LOGP_TOL, f"{label}.logp")
+    report[f"{label}_logp_mp_err"] = _close(got.logp_mp.cpu(), want.logp_mp, LOGP_TOL,
+                                            f"{label}.logp_mp", ok)
+    comp_want = np.where(want.member == 1, want.sum_safe_x / want.sum_safe, 1.0)
+    comp_want = np.where(np.isnan(want.logp), np.nan, comp_want)
+    _close(got.comp_mp.cpu(), comp_want, lambda w: 1e-6 + 1e-4 * np.abs(w), f"{label}.comp_mp", ok)
+    if got.mask is not None and want.mask is not None:
+        bits = unpack_mask(got.mask, V)
+        assert np.array_equal(bits[ok], want.mask[ok]), f"{label}.mask"
+
+
+def check_flags(flags: torch.Tensor, res, ids: np.ndarray, V: int, ok_rows=None):
+    f = flags.cpu().numpy()
+    want = (res.train.member.astype(np.uint8) * 1)
+    if res.infer is not None:
+        want = want | (res.infer.member.astype(np.uint8) * 2)
+    want = want | np.where(ids < 0, 64, 0).astype(np.uint8) | np.where(ids >= V, 128, 0).astype(np.uint8)
+    if ok_rows is None:
+        ok_rows = np.ones(len(f), dtype=bool)
+    assert np.array_equal(f[ok_rows], want[ok_rows]), "flags"
+
+
+def check_grad(grad: torch.Tensor, want: np.ndarray, report, rows=None, label="grad"):
+    u = UNIT_ROUNDOFF[grad.dtype]
+    got = grad.detach().cpu().to(torch.float64).numpy()
+    if rows is not None:
+        got, want = got[rows], want[rows]
+    assert np.isfinite(got).all(), "gradient holds a non-finite value"
+    err = got - want
+    num = np.sqrt((err * err).sum(axis=1))
+    den = np.sqrt((want * want).sum(axis=1))
+    both_zero = (den == 0) & (np.abs(got).sum(axis=1) == 0)
+    rel = np.where(both_zero, 0.0, num / np.maximum(den, 1e-300))
+    assert (rel <= GRAD_TOL + u).all(), f"{label}: worst row relative L2 {rel.max():.3e}"
+    assert (np.abs(err) <= (GRAD_TOL + u) * np.abs(want) + 1e-30).all(), f"{label}: element bound"
+    assert ((want == 0) <= (got == 0)).all(), f"{label}: pruned entries must be exactly zero"
+    report[f"{label}_worst_row_rel_l2"] = float(rel.max())
+    report[f"{label}_zero_rows"] = int(both_zero.sum())
+
+
+def check_forward(res_gpu, batch, rho, V, want_grad, report=None, threads=8):
+    """Full element-by-element comparison of one dvp_forward result."""
+    report = {} if report is None else report
+    want = run_oracle(batch.train, batch.infer, batch.ids, rho,
+                      upstream=batch.upstream if want_grad else None,
+                      want_mask=res_gpu.train.mask is not None, threads=threads)
+    check_side(res_gpu.train, want.train, batch.train, V, "train", report)
+    near = near_threshold_rows(batch.train, want.train)
+    if want.infer is not None:
+        check_side(res_gpu.infer, want.infer, batch.infer, V, "infer", report)
+        near = near | near_threshold_rows(batch.infer, want.infer)
+        report["log_ratio_err"] = _close(res_gpu.log_ratio.cpu(), want.log_ratio, LOGP_TOL,
+                                         "log_ratio", ~near)
+    check_flags(res_gpu.flags, want, batch.ids.cpu().numpy(), V, ~near)
+    if want_grad:
+        check_grad(res_gpu.grad_train, want.grad, report, rows=~near)
+    report["mean_safe_set_size"] = float(want.train.count.mean())
+    report["frac_sampled_in_train_set"] = float(want.train.member.mean())
+    return report, want
