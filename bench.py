@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the DVP hot path: pruned log-prob forward+backward tokens/s.
+
+A step is one pass of the whole hot path over one synthetic batch: one
+``dvp_forward`` call that reads the training and inference logits and writes
+the gradient (Def. 5.1, Def. 5.2, Prop. 5.4) for every token of the batch.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--rho R]
+  python bench.py --impl reference ...     # the fp64 CPU checker on host cores
+
+With N > 1 (launched by torchrun, one rank per GPU) every rank processes its
+own batch of the same shape: rows are independent, so there is no data-path
+collective, only the barrier and the max-over-ranks of the device time.
+Rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "pruned_logprob_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes per launch of the row kernel (dram__bytes_read.sum + dram__bytes_write.sum
+# from one ncu capture), keyed by workload; valid only for the kernel sources whose
+# digest is recorded with it, scaled by rows when the capture used fewer rows.
+NCU_TRAFFIC = {
+}
+
+
+def _kernel_digest() -> str:
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2512_23087_b200", "csrc")
+    for name in ("dvp_common.cuh", "dvp_rows.cu"):
+        h.update(open(os.path.join(csrc, name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smax, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            sm.sort()
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(smax), reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=max(power))
+        return out
+
+
+def _dist_setup():
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    return rank, world, local
+
+
+def _oracle_sample(host, rho, threads, want_grad):
+    """Time the fp64 checker on ``host`` (a dict of host arrays)."""
+    import oracle
+    t0 = time.perf_counter()
+    res = oracle.dvp_rows(host["train"], host["ids"], rho, dtype=host["dtype"], infer=host["infer"],
+                          upstream=host["upstream"] if want_grad else None, want_grad=want_grad,
+                          threads=threads)
+    return time.perf_counter() - t0, res.threads
+
+
+def _host_rows(batch, r0, r1):
+    import numpy as np
+    import torch
+    import oracle
+
+    def st(x):
+        x = x[r0:r1].cpu()
+        return x.numpy() if x.dtype == torch.float32 else x.view(torch.int16).numpy().view(np.uint16)
+    code = {torch.float32: oracle.F32, torch.bfloat16: oracle.BF16, torch.float16: oracle.F16}
+    return {"train": st(batch.train), "infer": st(batch.infer), "ids": batch.ids[r0:r1].cpu().numpy(),
+            "upstream": batch.upstream[r0:r1].cpu().numpy().astype("f8"),
+            "dtype": code[batch.train.dtype]}
+
+
+def cpu_baseline(batch, rho, backward):
+    """The checker as it stands, all host cores, on the first rows of the batch."""
+    cores = os.cpu_count() or 1
+    slab = 256
+    total_t, rows, used = 0.0, 0, 1
+    for i in range(16):
+        r0 = i * slab
+        if r0 + slab > batch.train.shape[0]:
+            break
+        dt, used = _oracle_sample(_host_rows(batch, r0, r0 + slab), rho, cores, backward)
+        total_t += dt
+        rows += slab
+        if total_t * used > 20.0:
+            break
+    return {"value": rows / total_t, "unit": UNIT, "cores": used, "kind": "oracle",
+            "sample": f"first {rows} rows of the batch (V={batch.train.shape[1]}), fp64, {used} threads, "
+                      f"rows split statically, {total_t:.2f} s wall"}
+
+
+def run_reference(args):
+    """--impl reference: the fp64 CPU checker, timed on host cores."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from paper_2512_23087_b200 import inputs
+    w = inputs.WORKLOADS[args.workload]
+    rho = args.rho if args.rho is not None else w.rhos[0]
+    rows_per_step = 128
+    batch = inputs.make_rows(w, seed=0, device="cpu", T=rows_per_step * 2, chunk_rows=64)
+    cores = os.cpu_count() or 1
+    host = [_host_rows(batch, i * rows_per_step, (i + 1) * rows_per_step) for i in range(2)]
+    for i in range(args.warmup):
+        _oracle_sample(host[i % 2], rho, cores, w.backward)
+    t, used = 0.0, 1
+    for i in range(args.steps):
+        dt, used = _oracle_sample(host[i % 2], rho, cores, w.backward)
+        t += dt
+    value = rows_per_step * args.steps / t
+    sample = (f"{rows_per_step} rows per step of {w.name} (V={w.V}, {w.dtype}), fp64 CPU checker, "
+              f"{used} threads")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": w.name, "T_per_step": rows_per_step, "V": w.V, "rho": rho,
+                   "logits_dtype": w.dtype, "note": "bounded sample of the workload per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def run_ours(args):
+    import torch
+    from paper_2512_23087_b200 import binding, inputs
+
+    rank, world, local = _dist_setup()
+    dev = torch.device("cuda", local)
+    w = inputs.WORKLOADS[args.workload]
+    rho = args.rho if args.rho is not None else w.rhos[0]
+    T = args.rows if args.rows else w.T
+    elem = 2 if w.dtype in ("bf16", "f16") else 4
+    grad_dtype = inputs.torch_dtype(w.grad_dtype or w.dtype)
+    grad_elem = torch.empty(0, dtype=grad_dtype).element_size()
+    batch = inputs.make_rows(w, seed=rank, device=dev, T=T)
+    V = batch.train.shape[1]
+    stream = torch.cuda.current_stream()
+
+    def step(out=None):
+        return binding.dvp_forward(batch.train, batch.ids, rho, infer_logits=batch.infer,
+                                   upstream=batch.upstream if w.backward else None,
+                                   grad_dtype=grad_dtype, stream=stream, launch_hint=args.launch_hint,
+                                   out=out)
+
+    warmup = max(args.warmup, 3)
+    res = step()
+    for _ in range(warmup - 1):
+        step(res)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+            torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step(res)
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop()
+    launches = args.steps          # one kernel per dvp_forward call
+
+    # ---- end to end: host buffers in, per-token results out, copies inside the timed region
+    slab = min(T, 2048)
+    n_slabs = (T + slab - 1) // slab
+    pool = 2
+    h_train = [torch.empty(slab, V, dtype=batch.train.dtype).pin_memory() for _ in range(pool)]
+    h_infer = [torch.empty(slab, V, dtype=batch.train.dtype).pin_memory() for _ in range(pool)]
+    for i in range(pool):
+        r0 = i * slab if (i + 1) * slab <= T else 0
+        h_train[i].copy_(batch.train[r0:r0 + slab])
+        h_infer[i].copy_(batch.infer[r0:r0 + slab])
+    h_ids = batch.ids.cpu().pin_memory()
+    h_up = batch.upstream.cpu().pin_memory()
+    h_out = torch.empty(3, T, dtype=torch.float32).pin_memory()
+    h_flags = torch.empty(T, dtype=torch.uint8).pin_memory()
+    d_train = [torch.empty(slab, V, dtype=batch.train.dtype, device=dev) for _ in range(2)]
+    d_infer = [torch.empty(slab, V, dtype=batch.train.dtype, device=dev) for _ in range(2)]
+    d_grad = [torch.empty(slab, V, dtype=grad_dtype, device=dev) for _ in range(2)]
+    copy_stream = torch.cuda.Stream(device=dev)
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+
+    def e2e_step():
+        d_ids = h_ids.to(dev, non_blocking=True)
+        d_up = h_up.to(dev, non_blocking=True)
+        ready = [torch.cuda.Event(), torch.cuda.Event()]
+        done = [None, None]
+        for s in range(n_slabs):
+            b = s % 2
+            rows = min(slab, T - s * slab)
+            with torch.cuda.stream(copy_stream):
+                if done[b] is not None:
+                    copy_stream.wait_event(done[b])
+                d_train[b][:rows].copy_(h_train[s % pool][:rows], non_blocking=True)
+                d_infer[b][:rows].copy_(h_infer[s % pool][:rows], non_blocking=True)
+                ready[b].record(copy_stream)
+            stream.wait_event(ready[b])
+            sl = slice(s * slab, s * slab + rows)
+            r = binding.dvp_forward(d_train[b][:rows], d_ids[sl], rho, infer_logits=d_infer[b][:rows],
+                                    upstream=d_up[sl] if w.backward else None,
+                                    grad_train=d_grad[b][:rows] if w.backward else None,
+                                    stream=stream, launch_hint=args.launch_hint)
+            h_out[0, sl].copy_(r.train.logp_mp, non_blocking=True)
+            h_out[1, sl].copy_(r.infer.logp_mp, non_blocking=True)
+            h_out[2, sl].copy_(r.log_ratio, non_blocking=True)
+            h_flags[sl].copy_(r.flags, non_blocking=True)
+            done[b] = torch.cuda.Event()
+            done[b].record(stream)
+
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    h2d = 2 * T * V * elem + T * 8 + T * 4
+    d2h = 3 * T * 4 + T
+
+    if world > 1:
+        t = torch.tensor([ms, e2e_s], device=dev, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms, e2e_s = t.tolist()
+    tokens = T * world
+    value = tokens * args.steps / (ms * 1e-3)
+    peak, peak_kind = _peaks()
+    alg_bytes = (2 * elem + (grad_elem if w.backward else 0)) * T * V
+    achieved = alg_bytes / (ms * 1e-3 / args.steps) / 1e9
+    traffic = None
+    rec = NCU_TRAFFIC.get(w.name)
+    if rec and rec.get("digest") == _kernel_digest() and rec.get("rho") == rho:
+        traffic = rec["bytes"] * (T / rec["T"])
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "T_per_gpu": T, "V": V, "logits_dtype": w.dtype,
+                   "grad_dtype": str(grad_dtype).replace("torch.", ""), "rho": rho,
+                   "backward": w.backward,
+                   "parallelism": f"rows sharded over {world} GPU(s), no collective",
+                   "l2": "inputs larger than L2, no flush" if alg_bytes > (1 << 30) else "inputs fit L2",
+                   "launch_hint": args.launch_hint},
+        "clocks": clocks,
+        "e2e": {"value": tokens * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                "note": f"pinned host slabs of {slab} rows, copies overlapped with kernels on a second "
+                        f"stream, per-token results copied back, gradient stays on the device"},
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                     "kernel": "dvp_row_kernel", "bytes_per_launch": alg_bytes,
+                     "frac_of_nominal_8TBs": achieved / 8000.0},
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(batch, rho, w.backward)
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_bf16_fwdbwd")
+    ap.add_argument("--rho", type=float, default=None)
+    ap.add_argument("--rows", type=int, default=0, help="override T (rows per GPU)")
+    ap.add_argument("--launch-hint", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -99,16 +99,18 @@ typedef struct {
  *                 -inf when a is outside V_S (importance ratio zero, remark
  *                 after Thm. 5.3), +inf when a is in V_S but outside V'_S
  *   flags         device [T] bytes, DVP_FLAG_* bits
- *   launch_hint   0 = library default; otherwise threads per block in the low
- *                 16 bits and loads in flight per thread in the next 8 bits
- *                 (tuning only, results do not depend on it)
+ *   launch_hint   0 = library default; otherwise threads per block (a multiple
+ *                 of 32, at most 512) in the low 16 bits and 16-byte loads in
+ *                 flight per thread (4 or 8) in the next 8 bits; tuning only,
+ *                 the safe set and counts do not depend on it
  *
  * Rows whose start is 16-byte aligned in all three matrices take the
  * vectorised kernels; any other layout takes a scalar kernel, same results.
  * Needs no workspace.  Errors: DVP_ERR_INVALID_ARG for NULL required
  * pointers, T < 0, V < 1, ld < V, rho outside [0,1] or NaN, upstream without
- * grad_train or the reverse; DVP_ERR_UNSUPPORTED for unknown dtypes or a row
- * too long for the on-chip row summary (V above about 1.7 million elements).
+ * grad_train or the reverse, a malformed launch_hint; DVP_ERR_UNSUPPORTED
+ * for unknown dtypes or V >= 2^31 - 256.  Rows too long for the on-chip row
+ * summary of the vectorised kernel fall back to the scalar kernel.
  * T = 0 is a valid no-op.
  */
 typedef struct {

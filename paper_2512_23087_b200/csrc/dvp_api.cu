@@ -9,7 +9,7 @@ bool dtype_ok(int d) { return d == DVP_F32 || d == DVP_BF16 || d == DVP_F16; }
 
 bool hint_ok(uint32_t hint) {
   const uint32_t threads = hint & 0xffff, unroll = (hint >> 16) & 0xff;
-  if (threads != 0 && (threads % 32 != 0 || threads > 1024)) return false;
+  if (threads != 0 && (threads % 32 != 0 || threads > 512)) return false;
   return unroll == 0 || unroll == 2 || unroll == 4 || unroll == 8;
 }
 

@@ -1,18 +1,20 @@
 """Comparison of the CUDA library's outputs with the fp64 oracle.
 
 Tolerances (stated once, used by every parity test):
-  * row max, safe-set size, membership flags, packed mask: bit-exact, except
-    rows that hold a logit within 1e-6 relative of the threshold, which are
-    counted and reported (the exact comparison scheme makes none expected);
+  * row max, safe-set size, membership flags, packed mask: bit-exact on every
+    row.  Rows that hold a logit within 1e-6 relative of the threshold are
+    counted and reported, but they get no allowance: the library decides
+    membership exactly as the double comparison does, so none is needed;
   * log-probabilities (logp, logp_mp, log_ratio): 1e-4 absolute, infinities
     and NaNs must coincide;
   * lse, lse_safe: 1e-4 absolute plus one float32 rounding of the value (they
     are float32 outputs whose magnitude can reach the hundreds);
   * gradients: per row, ||G - G_oracle||_2 <= (1e-3 + u) ||G_oracle||_2 with u
-    the unit roundoff of the gradient's storage type (0 for float32, 2^-9 for
-    bfloat16, 2^-12 for float16): round-to-nearest storage alone contributes
+    the unit roundoff of the gradient's storage type (0 for float32, 2^-8 for
+    bfloat16, 2^-11 for float16): round-to-nearest storage alone contributes
     up to u.  Rows where both are zero pass.  In addition every element must
-    sit within (1e-3 + u) |G_oracle| + 1e-30 of the oracle's element.
+    sit within (1e-3 + u) |G_oracle| + a of the oracle's element, a being half
+    the spacing of the storage type's subnormals (2^-25 for float16) or 1e-30.
 """
 from __future__ import annotations
 
@@ -23,7 +25,8 @@ import oracle
 
 LOGP_TOL = 1e-4
 GRAD_TOL = 1e-3
-UNIT_ROUNDOFF = {torch.float32: 0.0, torch.bfloat16: 2.0 ** -9, torch.float16: 2.0 ** -12}
+UNIT_ROUNDOFF = {torch.float32: 0.0, torch.bfloat16: 2.0 ** -8, torch.float16: 2.0 ** -11}
+SUBNORMAL_HALF_STEP = {torch.float32: 1e-30, torch.bfloat16: 1e-30, torch.float16: 2.0 ** -25}
 ORACLE_DTYPE = {torch.float32: oracle.F32, torch.bfloat16: oracle.BF16, torch.float16: oracle.F16}
 
 
@@ -83,7 +86,7 @@ def unpack_mask(mask: torch.Tensor, V: int) -> np.ndarray:
 def check_side(got, want, stored, V, label, report):
     """got: namespace of device tensors; want: oracle.Side."""
     near = near_threshold_rows(stored, want)
-    ok = ~near
+    ok = np.ones_like(near)
     report[f"{label}_near_threshold_rows"] = int(near.sum())
     assert np.array_equal(got.max.cpu().numpy().astype(np.float64), want.max), f"{label}.max"
     cnt = got.count.cpu().numpy().astype(np.int64)
@@ -127,9 +130,10 @@ def check_grad(grad: torch.Tensor, want: np.ndarray, report, rows=None, label="g
     both_zero = (den == 0) & (np.abs(got).sum(axis=1) == 0)
     rel = np.where(both_zero, 0.0, num / np.maximum(den, 1e-300))
     assert (rel <= GRAD_TOL + u).all(), f"{label}: worst row relative L2 {rel.max():.3e}"
-    assert (np.abs(err) <= (GRAD_TOL + u) * np.abs(want) + 1e-30).all(), f"{label}: element bound"
+    floor = SUBNORMAL_HALF_STEP[grad.dtype]
+    assert (np.abs(err) <= (GRAD_TOL + u) * np.abs(want) + floor).all(), f"{label}: element bound"
     assert ((want == 0) <= (got == 0)).all(), f"{label}: pruned entries must be exactly zero"
-    report[f"{label}_worst_row_rel_l2"] = float(rel.max())
+    report[f"{label}_worst_row_rel_l2"] = float(rel.max()) if rel.size else 0.0
     report[f"{label}_zero_rows"] = int(both_zero.sum())
 
 
@@ -145,10 +149,11 @@ def check_forward(res_gpu, batch, rho, V, want_grad, report=None, threads=8):
         check_side(res_gpu.infer, want.infer, batch.infer, V, "infer", report)
         near = near | near_threshold_rows(batch.infer, want.infer)
         report["log_ratio_err"] = _close(res_gpu.log_ratio.cpu(), want.log_ratio, LOGP_TOL,
-                                         "log_ratio", ~near)
-    check_flags(res_gpu.flags, want, batch.ids.cpu().numpy(), V, ~near)
+                                         "log_ratio")
+    report["near_threshold_rows"] = int(near.sum())
+    check_flags(res_gpu.flags, want, batch.ids.cpu().numpy(), V)
     if want_grad:
-        check_grad(res_gpu.grad_train, want.grad, report, rows=~near)
+        check_grad(res_gpu.grad_train, want.grad, report)
     report["mean_safe_set_size"] = float(want.train.count.mean())
     report["frac_sampled_in_train_set"] = float(want.train.member.mean())
     return report, want
