@@ -15,16 +15,16 @@
 
 namespace dvp {
 
-// One thread's chunk of sweep `i`: kUnroll 16-byte vectors, vector u at index
-// (i * kUnroll + u) * blockDim + tid, kept packed as loaded.  Elements past V
-// are filled with -inf.
+// A chunk: the kUnroll 16-byte vectors that thread `tid` loads in sweep step
+// `i`, vector u at index (i * kUnroll + u) * blockDim + tid, kept packed as
+// loaded.  Elements past V are filled with -inf.
 template <typename TIn, int kUnroll>
 struct Chunk {
   static constexpr int kPerVec = Storage<TIn>::kPerVec;
   uint4 raw[kUnroll];
 
-  __device__ __forceinline__ void load(const TIn *row, int V, int n_full, int vb) {
-    const int v0 = vb + threadIdx.x;
+  __device__ __forceinline__ void load(const TIn *row, int V, int n_full, int vb, int tid) {
+    const int v0 = vb + tid;
     if (vb + kUnroll * (int)blockDim.x <= n_full) {
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u)
@@ -51,22 +51,75 @@ struct Chunk {
   __device__ __forceinline__ void get(int u, float *x) const { Storage<TIn>::unpack(raw[u], x); }
 };
 
+// Chunks that can hold a safe token, per warp, in the order (sweep step, lane).
+// A warp whose chunks do not fit (a dense safe set) walks all of its chunks
+// instead, which is then the efficient thing to do anyway.
+constexpr int kHotCap = 128;
+
+struct HotList {
+  uint32_t *slots;  // kHotCap entries of this warp: step * 32 + lane
+  int count;        // chunks at or above the threshold (may exceed kHotCap)
+  __device__ __forceinline__ bool fits() const { return count <= kHotCap; }
+};
+
+__device__ __forceinline__ HotList build_hot_list(const float *chunk_max, int n_steps, float tau,
+                                                  uint32_t *hot_smem) {
+  const int lane = threadIdx.x & 31;
+  HotList h;
+  h.slots = hot_smem + (threadIdx.x >> 5) * kHotCap;
+  h.count = 0;
+  for (int i = 0; i < n_steps; ++i) {
+    const bool f = chunk_max[i * blockDim.x + threadIdx.x] >= tau;
+    const unsigned b = __ballot_sync(0xffffffffu, f);
+    if (f) {
+      const int pos = h.count + __popc(b & ((1u << lane) - 1u));
+      if (pos < kHotCap) h.slots[pos] = (uint32_t)(i * 32 + lane);
+    }
+    h.count += __popc(b);
+  }
+  __syncwarp();
+  return h;
+}
+
+// Contribution of one chunk to the masked sum and the count (Def. 5.2).
+template <typename TIn, int kUnroll>
+__device__ __forceinline__ void chunk_masked_sum(const Chunk<TIn, kUnroll> &c, int vb, int tid,
+                                                 int a, int va, float tau, float m, SumCount &sc) {
+  constexpr int kPerVec = Storage<TIn>::kPerVec;
+#pragma unroll
+  for (int u = 0; u < kUnroll; ++u) {
+    const int v = vb + u * (int)blockDim.x + tid;
+    float x[kPerVec];
+    c.get(u, x);
+    // the sampled token is left out so that 1 - pi^mp(a) has no cancellation
+    const int ja = v == va ? a - va * kPerVec : -1;
+#pragma unroll
+    for (int j = 0; j < kPerVec; ++j) {
+      if (x[j] >= tau) {
+        ++sc.n;
+        if (j != ja) sc.s += ex2((x[j] - m) * kLog2e);
+      }
+    }
+  }
+}
+
 // Sweeps 1 and 2 over one row: statistics of one side.
 template <typename TIn, int kUnroll>
 __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int a, double log_rho,
-                                               float *chunk_max, float *scratch,
-                                               uint32_t *mask_row) {
+                                               float *chunk_max, float *scratch, uint32_t *hot_smem,
+                                               HotList &hot, uint32_t *mask_row) {
   constexpr int kPerVec = Storage<TIn>::kPerVec;
   const int n_full = V / kPerVec;
   const int n_vec = (V + kPerVec - 1) / kPerVec;
   const int per_sweep = kUnroll * (int)blockDim.x;
-  const int n_sweeps = (n_vec + per_sweep - 1) / per_sweep;
+  const int n_steps = (n_vec + per_sweep - 1) / per_sweep;
+  const int tid = threadIdx.x;
 
   // ---- sweep 1: online max / sum-exp, chunk maxima to shared memory
   MaxSum acc = {kNegInf, 0.f};
-  for (int i = 0; i < n_sweeps; ++i) {
+  for (int i = 0; i < n_steps; ++i) {
     Chunk<TIn, kUnroll> c;
-    c.load(row, V, n_full, i * per_sweep);
+    c.load(row, V, n_full, i * per_sweep, tid);
     float cm = kNegInf;
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
@@ -75,7 +128,7 @@ __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int a, dou
 #pragma unroll
       for (int j = 0; j < kPerVec; ++j) cm = fmaxf(cm, x[j]);
     }
-    chunk_max[i * blockDim.x + threadIdx.x] = cm;
+    chunk_max[i * blockDim.x + tid] = cm;
     if (cm > kNegInf) {
       if (cm > acc.m) {
         acc.s *= ex2((acc.m - cm) * kLog2e);
@@ -106,24 +159,22 @@ __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int a, dou
   // ---- sweep 2: only chunks that can hold a safe token
   const int va = has_a ? a / kPerVec : -1;
   SumCount sc = {0.f, 0};
-  for (int i = 0; i < n_sweeps; ++i) {
-    if (chunk_max[i * blockDim.x + threadIdx.x] >= st.tau) {
+  hot = build_hot_list(chunk_max, n_steps, st.tau, hot_smem);
+  if (hot.fits()) {
+    const int wbase = tid & ~31;
+    for (int q = tid & 31; q < hot.count; q += 32) {
+      const uint32_t e = hot.slots[q];
+      const int vb = (int)(e >> 5) * per_sweep, owner = wbase + (int)(e & 31);
       Chunk<TIn, kUnroll> c;
-      c.load(row, V, n_full, i * per_sweep);
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        const int v = i * per_sweep + u * (int)blockDim.x + threadIdx.x;
-        float x[kPerVec];
-        c.get(u, x);
-        // the sampled token is left out so that 1 - pi^mp(a) has no cancellation
-        const int ja = v == va ? a - va * kPerVec : -1;
-#pragma unroll
-        for (int j = 0; j < kPerVec; ++j) {
-          if (x[j] >= st.tau) {
-            ++sc.n;
-            if (j != ja) sc.s += ex2((x[j] - st.m) * kLog2e);
-          }
-        }
+      c.load(row, V, n_full, vb, owner);
+      chunk_masked_sum<TIn, kUnroll>(c, vb, owner, a, va, st.tau, st.m, sc);
+    }
+  } else {
+    for (int i = 0; i < n_steps; ++i) {
+      if (chunk_max[i * blockDim.x + tid] >= st.tau) {
+        Chunk<TIn, kUnroll> c;
+        c.load(row, V, n_full, i * per_sweep, tid);
+        chunk_masked_sum<TIn, kUnroll>(c, i * per_sweep, tid, a, va, st.tau, st.m, sc);
       }
     }
   }
@@ -134,7 +185,7 @@ __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int a, dou
   // ---- optional packed membership mask (diagnostic output, plain loads)
   if (mask_row) {
     const int n_words = (V + 31) / 32;
-    for (int w = threadIdx.x; w < n_words; w += blockDim.x) {
+    for (int w = tid; w < n_words; w += blockDim.x) {
       uint32_t bits = 0;
       for (int b = 0; b < 32; ++b) {
         const long long k = (long long)w * 32 + b;
@@ -146,55 +197,90 @@ __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int a, dou
   return st;
 }
 
-// Sweep 3: gradient of g * ln pi^mp(a) over the row (Prop. 5.4, set fixed).
+// Gradient entries of one chunk (Prop. 5.4, set fixed), stored to the row.
+template <typename TIn, typename TGrad, int kUnroll>
+__device__ __forceinline__ void chunk_grad(const Chunk<TIn, kUnroll> &c, TGrad *grow, int V,
+                                           int n_full, int n_vec, int vb, int tid, int a, int va,
+                                           float tau, float m, float coef, float g_a) {
+  constexpr int kPerVec = Storage<TIn>::kPerVec;
+#pragma unroll
+  for (int u = 0; u < kUnroll; ++u) {
+    const int v = vb + u * (int)blockDim.x + tid;
+    if (v >= n_vec) continue;
+    float x[kPerVec], out[kPerVec];
+    c.get(u, x);
+    const int ja = v == va ? a - va * kPerVec : -1;
+#pragma unroll
+    for (int j = 0; j < kPerVec; ++j) {
+      out[j] = x[j] >= tau ? coef * ex2((x[j] - m) * kLog2e) : 0.f;
+      if (j == ja) out[j] = g_a;
+    }
+    if (v < n_full) {
+      store_grads<TGrad, kPerVec>(grow + (size_t)v * kPerVec, out);
+    } else {
+#pragma unroll
+      for (int j = 0; j < kPerVec; ++j) {
+        const long long k = (long long)v * kPerVec + j;
+        if (k < V) grow[k] = Storage<TGrad>::narrow(out[j]);
+      }
+    }
+  }
+}
+
+// Sweep 3: gradient of g * ln pi^mp(a) over the row.  Chunks without a safe
+// token are written as zeros without being read.
 template <typename TIn, typename TGrad, int kUnroll>
 __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int a,
-                                         const SideStats &st, float g, const float *chunk_max) {
+                                         const SideStats &st, float g, const float *chunk_max,
+                                         const HotList &hot) {
   constexpr int kPerVec = Storage<TIn>::kPerVec;
   const int n_full = V / kPerVec;
   const int n_vec = (V + kPerVec - 1) / kPerVec;
   const int per_sweep = kUnroll * (int)blockDim.x;
-  const int n_sweeps = (n_vec + per_sweep - 1) / per_sweep;
+  const int n_steps = (n_vec + per_sweep - 1) / per_sweep;
+  const int tid = threadIdx.x;
   const float s_safe = st.s_x + st.e_a;
   // a pruned or missing sampled token has weight zero: the row is all zeros
   const bool live = st.member;
   const float coef = live ? -g / s_safe : 0.f;
   const float g_a = live ? g * (st.s_x / s_safe) : 0.f;
-  const float tau = live ? st.tau : -kNegInf;  // +inf: nothing passes
   const int va = live ? a / kPerVec : -1;
+  const bool listed = live && hot.fits();
+  const float tau = live ? st.tau : -kNegInf;  // +inf: nothing passes
 
-  for (int i = 0; i < n_sweeps; ++i) {
+  for (int i = 0; i < n_steps; ++i) {
     const int vb = i * per_sweep;
-    const bool hot = chunk_max[i * blockDim.x + threadIdx.x] >= tau;
-    Chunk<TIn, kUnroll> c;
-    if (hot) c.load(row, V, n_full, vb);
+    if (chunk_max[i * blockDim.x + tid] >= tau) {
+      if (!listed) {
+        Chunk<TIn, kUnroll> c;
+        c.load(row, V, n_full, vb, tid);
+        chunk_grad<TIn, TGrad, kUnroll>(c, grow, V, n_full, n_vec, vb, tid, a, va, tau, st.m, coef,
+                                        g_a);
+      }
+      continue;
+    }
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
-      const int v = vb + u * (int)blockDim.x + threadIdx.x;
-      if (v >= n_vec) continue;
-      float out[kPerVec];
-      if (hot) {
-        float x[kPerVec];
-        c.get(u, x);
-        const int ja = v == va ? a - va * kPerVec : -1;
-#pragma unroll
-        for (int j = 0; j < kPerVec; ++j) {
-          out[j] = x[j] >= tau ? coef * ex2((x[j] - st.m) * kLog2e) : 0.f;
-          if (j == ja) out[j] = g_a;
-        }
-      } else {
-#pragma unroll
-        for (int j = 0; j < kPerVec; ++j) out[j] = 0.f;
-      }
+      const int v = vb + u * (int)blockDim.x + tid;
       if (v < n_full) {
-        store_grads<TGrad, kPerVec>(grow + (size_t)v * kPerVec, out);
-      } else {
-#pragma unroll
+        store_zeros<TGrad, kPerVec>(grow + (size_t)v * kPerVec);
+      } else if (v < n_vec) {
         for (int j = 0; j < kPerVec; ++j) {
           const long long k = (long long)v * kPerVec + j;
-          if (k < V) grow[k] = Storage<TGrad>::narrow(out[j]);
+          if (k < V) grow[k] = Storage<TGrad>::narrow(0.f);
         }
       }
+    }
+  }
+  if (listed) {
+    const int wbase = tid & ~31;
+    for (int q = tid & 31; q < hot.count; q += 32) {
+      const uint32_t e = hot.slots[q];
+      const int vb = (int)(e >> 5) * per_sweep, owner = wbase + (int)(e & 31);
+      Chunk<TIn, kUnroll> c;
+      c.load(row, V, n_full, vb, owner);
+      chunk_grad<TIn, TGrad, kUnroll>(c, grow, V, n_full, n_vec, vb, owner, a, va, tau, st.m, coef,
+                                      g_a);
     }
   }
 }
@@ -202,8 +288,9 @@ __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int
 template <typename TIn, typename TGrad, int kUnroll>
 __global__ void __launch_bounds__(512, 2) dvp_row_kernel(const RowParams p) {
   extern __shared__ __align__(16) float smem[];
-  float *scratch = smem;         // 64 floats for the block reductions
-  float *chunk_max = smem + 64;  // one float per (sweep, thread)
+  float *scratch = smem;  // 64 floats for the block reductions
+  uint32_t *hot_smem = reinterpret_cast<uint32_t *>(smem + 64);  // kHotCap per warp
+  float *chunk_max = smem + 64 + (blockDim.x >> 5) * kHotCap;    // one float per (step, thread)
 
   const long long t = blockIdx.x;
   const long long id = p.ids ? load_id(p.ids, p.id_is_i32, t) : -1;
@@ -213,20 +300,23 @@ __global__ void __launch_bounds__(512, 2) dvp_row_kernel(const RowParams p) {
 
   const TIn *trow = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
   uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * ((p.V + 31) / 32) : nullptr;
-  const SideStats st = row_stats<TIn, kUnroll>(trow, V, a, p.log_rho, chunk_max, scratch, mask_t);
+  HotList hot;
+  const SideStats st =
+      row_stats<TIn, kUnroll>(trow, V, a, p.log_rho, chunk_max, scratch, hot_smem, hot, mask_t);
 
   if (p.grad) {
     const float g = p.upstream[t];
-    row_grad<TIn, TGrad, kUnroll>(trow, reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad, V, a,
-                                  st, g, chunk_max);
+    row_grad<TIn, TGrad, kUnroll>(trow, reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad, V, a, st,
+                                  g, chunk_max, hot);
   }
 
   SideStats si;
   if (p.infer) {
-    __syncthreads();  // chunk_max is reused for the second matrix
+    __syncthreads();  // chunk_max and the hot lists are reused for the second matrix
     const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
     uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
-    si = row_stats<TIn, kUnroll>(irow, V, a, p.log_rho, chunk_max, scratch, mask_i);
+    HotList hot_i;
+    si = row_stats<TIn, kUnroll>(irow, V, a, p.log_rho, chunk_max, scratch, hot_smem, hot_i, mask_i);
   }
 
   if (threadIdx.x == 0) {
@@ -370,7 +460,7 @@ __global__ void dvp_backward_kernel(const BackwardParams p) {
     const int va = live ? (int)(a / kPerVec) : -1;
     for (int vb = 0; vb < n_vec; vb += per_sweep) {
       Chunk<TIn, kUnroll> c;
-      c.load(row, V, n_full, vb);
+      c.load(row, V, n_full, vb, threadIdx.x);
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
         const int v = vb + u * (int)blockDim.x + threadIdx.x;
@@ -433,12 +523,12 @@ static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s
   while (threads > 64 && (long long)threads * unroll / 2 >= n_vec) threads /= 2;
   auto smem_for = [&](int u) {
     const long long per = (long long)u * threads;
-    return (size_t)(64 + ((n_vec + per - 1) / per) * threads) * sizeof(float);
+    return (size_t)(64 + (threads / 32) * kHotCap + ((n_vec + per - 1) / per) * threads) * sizeof(float);
   };
   const size_t smem_cap = 200 * 1024;
   if (vec_ok) {
     if (unroll < 4) unroll = 4;
-    while (unroll < 8 && smem_for(unroll) > 64 * 1024) unroll *= 2;
+    while (unroll < 8 && smem_for(unroll) > 72 * 1024) unroll *= 2;
     if (smem_for(unroll) <= smem_cap) {
       if (unroll <= 4) return launch_rows_vec<TIn, TGrad, 4>(p, threads, smem_for(4), s);
       return launch_rows_vec<TIn, TGrad, 8>(p, threads, smem_for(8), s);
