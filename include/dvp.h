@@ -100,11 +100,11 @@ typedef struct {
  *                 after Thm. 5.3), +inf when a is in V_S but outside V'_S
  *   flags         device [T] bytes, DVP_FLAG_* bits
  *   launch_hint   0 = library default; otherwise threads per block (a multiple
- *                 of 32, at most 512) in the low 16 bits and 16-byte loads in
- *                 flight per thread (4 or 8) in the next 8 bits; tuning only,
- *                 the safe set and counts do not depend on it
+ *                 of 32, at most 512) in the low 16 bits and 32-byte loads per
+ *                 thread and pipeline stage (1, 2 or 4) in the next 8 bits;
+ *                 tuning only, the safe set and counts do not depend on it
  *
- * Rows whose start is 16-byte aligned in all three matrices take the
+ * Rows whose start is 32-byte aligned in all three matrices take the
  * vectorised kernels; any other layout takes a scalar kernel, same results.
  * Needs no workspace.  Errors: DVP_ERR_INVALID_ARG for NULL required
  * pointers, T < 0, V < 1, ld < V, rho outside [0,1] or NaN, upstream without

@@ -8,9 +8,9 @@ namespace {
 bool dtype_ok(int d) { return d == DVP_F32 || d == DVP_BF16 || d == DVP_F16; }
 
 bool hint_ok(uint32_t hint) {
-  const uint32_t threads = hint & 0xffff, unroll = (hint >> 16) & 0xff;
+  const uint32_t threads = hint & 0xffff, stage = (hint >> 16) & 0xff;
   if (threads != 0 && (threads % 32 != 0 || threads > 512)) return false;
-  return unroll == 0 || unroll == 2 || unroll == 4 || unroll == 8;
+  return stage == 0 || stage == 1 || stage == 2 || stage == 4;
 }
 
 bool side_empty(const dvp_side_out &o) {

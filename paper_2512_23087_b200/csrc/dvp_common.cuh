@@ -30,11 +30,24 @@ __device__ __forceinline__ uint4 ld_stream16(const void *p) {
   return v;
 }
 
+// 32-byte variant: one DRAM sector per lane and instruction.
+__device__ __forceinline__ void ld_stream32(const void *p, uint32_t (&w)[8]) {
+  asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]),
+                 "=r"(w[7])
+               : "l"(p));
+}
+
 // Streaming stores (evict-first): the gradient is written once and not read
 // again by this library.
 __device__ __forceinline__ void st_stream16(void *p, uint4 v) {
   asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
                "r"(v.w)
+               : "memory");
+}
+__device__ __forceinline__ void st_stream32(void *p, const uint32_t (&w)[8]) {
+  asm volatile("st.global.cs.v8.u32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]),
+               "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
                : "memory");
 }
 __device__ __forceinline__ void st_stream8(void *p, uint2 v) {
@@ -177,6 +190,66 @@ __device__ __forceinline__ MaxSum block_reduce_maxsum(MaxSum v, float *scratch) 
   return r;
 }
 
+// Log-sum-exp state kept in the base-2 domain so that each term costs one FMA
+// and one ex2: with l = kLog2e (a float), the elements seen so far satisfy
+//   sum_k 2^{z_k l} = 2^c s,   c = fl(m l),   m = their maximum.
+struct LogSum {
+  float m, c, s;
+};
+
+__device__ __forceinline__ LogSum combine(LogSum a, LogSum b) {
+  LogSum r;
+  r.m = fmaxf(a.m, b.m);
+  r.c = fmaxf(a.c, b.c);
+  const float sa = a.c > kNegInf ? a.s * ex2(a.c - r.c) : 0.f;
+  const float sb = b.c > kNegInf ? b.s * ex2(b.c - r.c) : 0.f;
+  r.s = sa + sb;
+  return r;
+}
+
+// scratch: 96 floats of shared memory.  Result valid in every thread.
+__device__ __forceinline__ LogSum block_reduce_logsum(LogSum v, float *scratch) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    LogSum other;
+    other.m = __shfl_xor_sync(0xffffffffu, v.m, o);
+    other.c = __shfl_xor_sync(0xffffffffu, v.c, o);
+    other.s = __shfl_xor_sync(0xffffffffu, v.s, o);
+    v = (lane & o) ? combine(other, v) : combine(v, other);
+  }
+  __syncthreads();
+  if (lane == 0) {
+    scratch[warp] = v.m;
+    scratch[32 + warp] = v.c;
+    scratch[64 + warp] = v.s;
+  }
+  __syncthreads();
+  LogSum r;
+  r.m = lane < nwarp ? scratch[lane] : kNegInf;
+  r.c = lane < nwarp ? scratch[32 + lane] : kNegInf;
+  r.s = lane < nwarp ? scratch[64 + lane] : 0.f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    LogSum other;
+    other.m = __shfl_xor_sync(0xffffffffu, r.m, o);
+    other.c = __shfl_xor_sync(0xffffffffu, r.c, o);
+    other.s = __shfl_xor_sync(0xffffffffu, r.s, o);
+    r = (lane & o) ? combine(other, r) : combine(r, other);
+  }
+  return r;
+}
+
+// ln sum_k e^{z_k} from the base-2 state.  2^{z l} = e^{z lambda} with
+// lambda = l ln 2 = 1 - 1.3e-8, so ln sum e^{z} = ln 2 (c + log2 s) +
+// (1 - lambda) E[z], the mean taken under the softmax weights; the maximum
+// stands in for it (they differ by at most about ln V, times 1.3e-8).
+__device__ __forceinline__ double lse_from_logsum(const LogSum &v) {
+  const double ln2 = 0.6931471805599453094;
+  const double one_minus_lambda = 1.0 - (double)kLog2e * ln2;
+  return ln2 * ((double)v.c + (double)log2f(v.s)) + one_minus_lambda * (double)v.m;
+}
+
 struct SumCount {
   float s;
   int n;
@@ -239,8 +312,8 @@ __device__ __forceinline__ float threshold_f32(float m, double log_rho) {
 // Everything one side of one row reduces to.
 struct SideStats {
   float m;       // row max
-  float s;       // sum_k e^{z_k - m}
-  float s_x;     // sum over the safe set without the sampled token
+  double lse;    // ln sum_k e^{z_k}
+  float s_x;     // sum over the safe set of e^{z_k - m}, without the sampled token
   float e_a;     // e^{z_a - m} when a is in the safe set, else 0
   float z_a;     // logit of the sampled token (0 when there is none)
   float tau;     // threshold_f32(m, log_rho)
@@ -252,17 +325,17 @@ struct SideStats {
 __device__ __forceinline__ float finish_side(const dvp_side_out &o, long long t, const SideStats &st,
                                              bool has_id, bool bad_id) {
   const float s_safe = st.s_x + st.e_a;
-  const float log_s = logf(st.s), log_ss = logf(s_safe);
+  const float log_ss = logf(s_safe);
   const float nan = __int_as_float(0x7fc00000);
   float logp = nan, logp_mp = nan, comp = nan;
   if (has_id) {
-    logp = (st.z_a - st.m) - log_s;
+    logp = (float)((double)st.z_a - st.lse);
     logp_mp = st.member ? (st.z_a - st.m) - log_ss : kNegInf;
     comp = st.member ? st.s_x / s_safe : 1.f;
   }
   if (bad_id) logp = logp_mp = comp = nan;
   if (o.max) o.max[t] = st.m;
-  if (o.lse) o.lse[t] = st.m + log_s;
+  if (o.lse) o.lse[t] = (float)st.lse;
   if (o.lse_safe) o.lse_safe[t] = st.m + log_ss;
   if (o.logp) o.logp[t] = logp;
   if (o.logp_mp) o.logp_mp[t] = logp_mp;
@@ -289,8 +362,8 @@ struct BackwardParams {
   int id_is_i32;
 };
 
-// Launchers (dvp_rows.cu).  `hint`: threads per block in the low 16 bits, loads
-// in flight per thread in the next 8 bits, 0 = default.
+// Launchers (dvp_rows.cu).  `hint`: threads per block in the low 16 bits,
+// 32-byte loads per thread and pipeline stage in the next 8 bits, 0 = default.
 cudaError_t launch_row_kernels(const RowParams &p, int logits_dtype, int grad_dtype, uint32_t hint,
                                cudaStream_t s);
 cudaError_t launch_backward_kernel(const BackwardParams &p, int logits_dtype, int grad_dtype,

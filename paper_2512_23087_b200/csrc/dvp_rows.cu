@@ -1,75 +1,159 @@
 // Row kernels of Dynamic Vocabulary Pruning for sm_100a.
 //
 // One thread block owns one token row.  The row is streamed from HBM once
-// (sweep 1).  While it streams, every thread keeps an online log-sum-exp of
-// what it has seen and leaves in shared memory the maximum of each chunk it
-// loaded (a chunk = kUnroll 16-byte vectors of one thread).  Once the row
-// maximum, hence the threshold of Def. 5.1, is known, only the chunks whose
-// maximum reaches the threshold can hold safe tokens: sweep 2 (masked sum and
-// count, Def. 5.2) and sweep 3 (gradient, Prop. 5.4) revisit just those,
-// normally out of L2, and sweep 3 writes zeros for all the others without
-// reading anything.  With a sparse safe set the row costs one HBM read per
-// logit matrix and one HBM write of the gradient; with a dense safe set the
-// same code degrades to three sweeps, still correct.
+// (sweep 1) in 32-byte granules, one DRAM sector per lane and load, two
+// pipeline stages deep.  While it streams, every thread keeps an online
+// log-sum-exp of what it has seen and leaves in shared memory an upper bound
+// (bfloat16, rounded up) of the maximum of each granule it loaded.  Once the
+// row maximum, hence the threshold of Def. 5.1, is known, only granules whose
+// bound reaches the threshold can hold safe tokens: sweep 2 (masked sum and
+// count, Def. 5.2) and sweep 3 (gradient, Prop. 5.4) revisit just those, and
+// sweep 3 writes zeros for all the others without reading anything.  With a
+// sparse safe set a row costs one HBM read per logit matrix and one HBM write
+// of the gradient; with a dense safe set the same code degrades to three
+// sweeps, still correct.
 #include "dvp_common.cuh"
 
 namespace dvp {
 
-// A chunk: the kUnroll 16-byte vectors that thread `tid` loads in sweep step
-// `i`, vector u at index (i * kUnroll + u) * blockDim + tid, kept packed as
-// loaded.  Elements past V are filled with -inf.
-template <typename TIn, int kUnroll>
-struct Chunk {
-  static constexpr int kPerVec = Storage<TIn>::kPerVec;
-  uint4 raw[kUnroll];
+template <typename T>
+struct Pair;
+template <>
+struct Pair<__nv_bfloat16> {
+  using type = __nv_bfloat162;
+};
+template <>
+struct Pair<__half> {
+  using type = __half2;
+};
 
-  __device__ __forceinline__ void load(const TIn *row, int V, int n_full, int vb, int tid) {
-    const int v0 = vb + tid;
-    if (vb + kUnroll * (int)blockDim.x <= n_full) {
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u)
-        raw[u] = ld_stream16(row + (size_t)(v0 + u * (int)blockDim.x) * kPerVec);
+// ---- a 32-byte granule of a row, kept packed as loaded ------------------------
+
+template <typename TIn>
+struct Granule {
+  static constexpr int kElems = 32 / (int)sizeof(TIn);
+  uint32_t w[8];
+
+  __device__ __forceinline__ void load(const TIn *p) { ld_stream32(p, w); }
+
+  // Granule `g` of a row of V elements; elements past V read as -inf.
+  __device__ __forceinline__ void load_any(const TIn *row, int V, int n_full, int g) {
+    if (g < n_full) {
+      load(row + (size_t)g * kElems);
     } else {
+      __align__(16) TIn tmp[kElems];
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        const int v = v0 + u * (int)blockDim.x;
-        if (v < n_full) {
-          raw[u] = ld_stream16(row + (size_t)v * kPerVec);
-        } else {
-          __align__(16) TIn tmp[kPerVec];
-#pragma unroll
-          for (int j = 0; j < kPerVec; ++j) {
-            const long long k = (long long)v * kPerVec + j;
-            tmp[j] = k < V ? row[k] : Storage<TIn>::narrow(kNegInf);
-          }
-          raw[u] = *reinterpret_cast<const uint4 *>(tmp);
-        }
+      for (int j = 0; j < kElems; ++j) {
+        const long long k = (long long)g * kElems + j;
+        tmp[j] = k < V ? row[k] : Storage<TIn>::narrow(kNegInf);
       }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) w[i] = reinterpret_cast<const uint32_t *>(tmp)[i];
     }
   }
 
-  __device__ __forceinline__ void get(int u, float *x) const { Storage<TIn>::unpack(raw[u], x); }
+  __device__ __forceinline__ void get(float *x) const {
+    constexpr int kHalf = kElems / 2;
+    Storage<TIn>::unpack(make_uint4(w[0], w[1], w[2], w[3]), x);
+    Storage<TIn>::unpack(make_uint4(w[4], w[5], w[6], w[7]), x + kHalf);
+  }
+
+  __device__ __forceinline__ float max() const {
+    if constexpr (sizeof(TIn) == 4) {
+      float m = __uint_as_float(w[0]);
+#pragma unroll
+      for (int i = 1; i < 8; ++i) m = fmaxf(m, __uint_as_float(w[i]));
+      return m;
+    } else {
+      // packed two-at-a-time maxima, then the two halves of the last pair
+      using T2 = typename Pair<TIn>::type;
+      T2 p[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) p[i] = *reinterpret_cast<const T2 *>(&w[i]);
+#pragma unroll
+      for (int s = 4; s > 0; s >>= 1)
+#pragma unroll
+        for (int i = 0; i < s; ++i) p[i] = __hmax2(p[i], p[i + s]);
+      return fmaxf(Storage<TIn>::widen(p[0].x), Storage<TIn>::widen(p[0].y));
+    }
+  }
 };
 
-// Chunks that can hold a safe token, per warp, in the order (sweep step, lane).
-// A warp whose chunks do not fit (a dense safe set) walks all of its chunks
-// instead, which is then the efficient thing to do anyway.
-constexpr int kHotCap = 128;
+// Upper bound of a float as a bfloat16 bit pattern (round toward +inf).
+__device__ __forceinline__ uint16_t bf16_bits_round_up(float v) {
+  const uint32_t b = __float_as_uint(v);
+  // positive: bump the magnitude unless the low half is zero; negative: truncate
+  return (uint16_t)(((b & 0x80000000u) ? b : b + 0xffffu) >> 16);
+}
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
+  return __uint_as_float((uint32_t)b << 16);
+}
+
+template <typename TGrad, int kElems>
+__device__ __forceinline__ void store_granule(TGrad *dst, const float *out) {
+  constexpr int kBytes = kElems * (int)sizeof(TGrad);
+  if constexpr (sizeof(TGrad) == 4) {
+#pragma unroll
+    for (int i = 0; i < kElems; i += 8) {
+      uint32_t w[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) w[j] = __float_as_uint(out[i + j]);
+      st_stream32(dst + i, w);
+    }
+  } else {
+    uint32_t w[kElems / 2];
+#pragma unroll
+    for (int i = 0; i < kElems / 2; ++i) {
+      TGrad lo = Storage<TGrad>::narrow(out[2 * i]), hi = Storage<TGrad>::narrow(out[2 * i + 1]);
+      w[i] = (uint32_t) * reinterpret_cast<uint16_t *>(&lo) |
+             ((uint32_t) * reinterpret_cast<uint16_t *>(&hi) << 16);
+    }
+    if constexpr (kBytes == 32) {
+      uint32_t v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = w[i];
+      st_stream32(dst, v);
+    } else {
+      static_assert(kBytes == 16, "granule of 8 floats stored as 8 halves");
+      st_stream16(dst, make_uint4(w[0], w[1], w[2], w[3]));
+    }
+  }
+}
+
+template <typename TGrad, int kElems>
+__device__ __forceinline__ void store_zero_granule(TGrad *dst) {
+  constexpr int kBytes = kElems * (int)sizeof(TGrad);
+  const uint32_t z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  if constexpr (kBytes == 64) {
+    st_stream32(dst, z);
+    st_stream32(reinterpret_cast<char *>(dst) + 32, z);
+  } else if constexpr (kBytes == 32) {
+    st_stream32(dst, z);
+  } else {
+    st_stream16(dst, make_uint4(0, 0, 0, 0));
+  }
+}
+
+// ---- granules that can hold a safe token ----------------------------------------
+// Per warp, in the order (slot, lane): entry = ordinal of the granule among the
+// warp's granules.  A warp whose hot granules do not fit (a dense safe set)
+// walks all of its granules instead, which is then the efficient thing to do.
+constexpr int kHotCap = 256;
 
 struct HotList {
-  uint32_t *slots;  // kHotCap entries of this warp: step * 32 + lane
-  int count;        // chunks at or above the threshold (may exceed kHotCap)
+  uint32_t *slots;
+  int count;  // granules at or above the threshold (may exceed kHotCap)
   __device__ __forceinline__ bool fits() const { return count <= kHotCap; }
 };
 
-__device__ __forceinline__ HotList build_hot_list(const float *chunk_max, int n_steps, float tau,
+__device__ __forceinline__ HotList build_hot_list(const uint16_t *bound, int n_slots, float tau,
                                                   uint32_t *hot_smem) {
   const int lane = threadIdx.x & 31;
   HotList h;
   h.slots = hot_smem + (threadIdx.x >> 5) * kHotCap;
   h.count = 0;
-  for (int i = 0; i < n_steps; ++i) {
-    const bool f = chunk_max[i * blockDim.x + threadIdx.x] >= tau;
+  for (int i = 0; i < n_slots; ++i) {
+    const bool f = bf16_bits_to_float(bound[i * blockDim.x + threadIdx.x]) >= tau;
     const unsigned b = __ballot_sync(0xffffffffu, f);
     if (f) {
       const int pos = h.count + __popc(b & ((1u << lane) - 1u));
@@ -81,100 +165,159 @@ __device__ __forceinline__ HotList build_hot_list(const float *chunk_max, int n_
   return h;
 }
 
-// Contribution of one chunk to the masked sum and the count (Def. 5.2).
-template <typename TIn, int kUnroll>
-__device__ __forceinline__ void chunk_masked_sum(const Chunk<TIn, kUnroll> &c, int vb, int tid,
-                                                 int a, int va, float tau, float m, SumCount &sc) {
-  constexpr int kPerVec = Storage<TIn>::kPerVec;
+// Contribution of one granule to the masked sum and the count (Def. 5.2).
+template <typename TIn>
+__device__ __forceinline__ void granule_masked_sum(const Granule<TIn> &gr, int g, int a, float tau,
+                                                   float m, SumCount &sc) {
+  constexpr int kElems = Granule<TIn>::kElems;
+  float x[kElems];
+  gr.get(x);
+  // the sampled token is left out so that 1 - pi^mp(a) has no cancellation
+  const int ja = a - g * kElems;  // in [0, kElems) only inside the owner granule
 #pragma unroll
-  for (int u = 0; u < kUnroll; ++u) {
-    const int v = vb + u * (int)blockDim.x + tid;
-    float x[kPerVec];
-    c.get(u, x);
-    // the sampled token is left out so that 1 - pi^mp(a) has no cancellation
-    const int ja = v == va ? a - va * kPerVec : -1;
-#pragma unroll
-    for (int j = 0; j < kPerVec; ++j) {
-      if (x[j] >= tau) {
-        ++sc.n;
-        if (j != ja) sc.s += ex2((x[j] - m) * kLog2e);
-      }
+  for (int j = 0; j < kElems; ++j) {
+    if (x[j] >= tau) {
+      ++sc.n;
+      if (j != ja) sc.s += ex2((x[j] - m) * kLog2e);
     }
   }
 }
 
-// Sweeps 1 and 2 over one row: statistics of one side.
-template <typename TIn, int kUnroll>
-__device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int a, double log_rho,
-                                               float *chunk_max, float *scratch, uint32_t *hot_smem,
-                                               HotList &hot, uint32_t *mask_row) {
-  constexpr int kPerVec = Storage<TIn>::kPerVec;
-  const int n_full = V / kPerVec;
-  const int n_vec = (V + kPerVec - 1) / kPerVec;
-  const int per_sweep = kUnroll * (int)blockDim.x;
-  const int n_steps = (n_vec + per_sweep - 1) / per_sweep;
-  const int tid = threadIdx.x;
-
-  // ---- sweep 1: online max / sum-exp, chunk maxima to shared memory
-  MaxSum acc = {kNegInf, 0.f};
-  for (int i = 0; i < n_steps; ++i) {
-    Chunk<TIn, kUnroll> c;
-    c.load(row, V, n_full, i * per_sweep, tid);
-    float cm = kNegInf;
+// Gradient entries of one granule (Prop. 5.4, set fixed), stored to the row.
+template <typename TIn, typename TGrad>
+__device__ __forceinline__ void granule_grad(const Granule<TIn> &gr, TGrad *grow, int V, int n_full,
+                                             int g, int a, float tau, float m, float coef,
+                                             float g_a) {
+  constexpr int kElems = Granule<TIn>::kElems;
+  float x[kElems], out[kElems];
+  gr.get(x);
+  const int ja = a - g * kElems;
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      float x[kPerVec];
-      c.get(u, x);
+  for (int j = 0; j < kElems; ++j) {
+    out[j] = x[j] >= tau ? coef * ex2((x[j] - m) * kLog2e) : 0.f;
+    if (j == ja) out[j] = g_a;
+  }
+  if (g < n_full) {
+    store_granule<TGrad, kElems>(grow + (size_t)g * kElems, out);
+  } else {
 #pragma unroll
-      for (int j = 0; j < kPerVec; ++j) cm = fmaxf(cm, x[j]);
-    }
-    chunk_max[i * blockDim.x + tid] = cm;
-    if (cm > kNegInf) {
-      if (cm > acc.m) {
-        acc.s *= ex2((acc.m - cm) * kLog2e);
-        acc.m = cm;
-      }
-      float part = 0.f;
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        float x[kPerVec];
-        c.get(u, x);
-#pragma unroll
-        for (int j = 0; j < kPerVec; ++j) part += ex2((x[j] - acc.m) * kLog2e);
-      }
-      acc.s += part;
+    for (int j = 0; j < kElems; ++j) {
+      const long long k = (long long)g * kElems + j;
+      if (k < V) grow[k] = Storage<TGrad>::narrow(out[j]);
     }
   }
-  const MaxSum all = block_reduce_maxsum(acc, scratch);
+}
+
+// One pipeline stage of sweep 1: kStage granules of this thread.
+template <typename TIn, int kStage>
+struct Stage {
+  Granule<TIn> g[kStage];
+  __device__ __forceinline__ void load(const TIn *row, int V, int n_full, int step) {
+    const int g0 = step * kStage * (int)blockDim.x + threadIdx.x;
+    if ((step + 1) * kStage * (int)blockDim.x <= n_full) {
+#pragma unroll
+      for (int u = 0; u < kStage; ++u)
+        g[u].load(row + (size_t)(g0 + u * (int)blockDim.x) * Granule<TIn>::kElems);
+    } else {
+#pragma unroll
+      for (int u = 0; u < kStage; ++u) g[u].load_any(row, V, n_full, g0 + u * (int)blockDim.x);
+    }
+  }
+};
+
+template <typename TIn, int kStage>
+__device__ __forceinline__ void absorb_stage(const Stage<TIn, kStage> &st, int step, LogSum &acc,
+                                             uint16_t *bound) {
+  constexpr int kElems = Granule<TIn>::kElems;
+  float cm = kNegInf;
+#pragma unroll
+  for (int u = 0; u < kStage; ++u) {
+    const float gm = st.g[u].max();
+    bound[(step * kStage + u) * blockDim.x + threadIdx.x] = bf16_bits_round_up(gm);
+    cm = fmaxf(cm, gm);
+  }
+  if (cm > kNegInf) {
+    if (cm > acc.m) {
+      const float cn = cm * kLog2e;
+      acc.s *= ex2(acc.c - cn);  // acc.c = -inf at the start: the factor is 0
+      acc.m = cm;
+      acc.c = cn;
+    }
+    const float neg_c = -acc.c;
+    float part = 0.f;
+#pragma unroll
+    for (int u = 0; u < kStage; ++u) {
+      float x[kElems];
+      st.g[u].get(x);
+#pragma unroll
+      for (int j = 0; j < kElems; ++j) part += ex2(fmaf(x[j], kLog2e, neg_c));
+    }
+    acc.s += part;
+  }
+}
+
+// Sweeps 1 and 2 over one row: statistics of one side.
+template <typename TIn, int kStage>
+__device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int a, double log_rho,
+                                               uint16_t *bound, float *scratch, uint32_t *hot_smem,
+                                               HotList &hot, uint32_t *mask_row) {
+  constexpr int kElems = Granule<TIn>::kElems;
+  const int n_full = V / kElems;
+  const int n_gran = (V + kElems - 1) / kElems;
+  const int per_step = kStage * (int)blockDim.x;
+  const int n_steps = (n_gran + per_step - 1) / per_step;
+  const int tid = threadIdx.x;
+
+  // ---- sweep 1, two stages in flight
+  LogSum acc = {kNegInf, kNegInf, 0.f};
+  {
+    Stage<TIn, kStage> s0, s1;
+    s0.load(row, V, n_full, 0);
+    int step = 0;
+    for (; step + 1 < n_steps; step += 2) {
+      s1.load(row, V, n_full, step + 1);
+      absorb_stage<TIn, kStage>(s0, step, acc, bound);
+      if (step + 2 < n_steps) s0.load(row, V, n_full, step + 2);
+      absorb_stage<TIn, kStage>(s1, step + 1, acc, bound);
+    }
+    if (step < n_steps) absorb_stage<TIn, kStage>(s0, step, acc, bound);
+  }
+  const LogSum all = block_reduce_logsum(acc, scratch);
 
   SideStats st;
   st.m = all.m;
-  st.s = all.s;
+  st.lse = lse_from_logsum(all);
   st.tau = threshold_f32(all.m, log_rho);
   const bool has_a = a >= 0 && a < V;
   st.z_a = has_a ? Storage<TIn>::widen(row[a]) : 0.f;
   st.member = has_a && st.z_a >= st.tau;
   st.e_a = st.member ? ex2((st.z_a - st.m) * kLog2e) : 0.f;
 
-  // ---- sweep 2: only chunks that can hold a safe token
-  const int va = has_a ? a / kPerVec : -1;
+  // ---- sweep 2: only granules that can hold a safe token
   SumCount sc = {0.f, 0};
-  hot = build_hot_list(chunk_max, n_steps, st.tau, hot_smem);
+  const int n_slots = n_steps * kStage;  // granules per thread
+  hot = build_hot_list(bound, n_slots, st.tau, hot_smem);
   if (hot.fits()) {
-    const int wbase = tid & ~31;
-    for (int q = tid & 31; q < hot.count; q += 32) {
-      const uint32_t e = hot.slots[q];
-      const int vb = (int)(e >> 5) * per_sweep, owner = wbase + (int)(e & 31);
-      Chunk<TIn, kUnroll> c;
-      c.load(row, V, n_full, vb, owner);
-      chunk_masked_sum<TIn, kUnroll>(c, vb, owner, a, va, st.tau, st.m, sc);
+    const int wbase = tid & ~31, lane = tid & 31;
+    for (int q = lane; q < hot.count; q += 64) {
+      const uint32_t e0 = hot.slots[q];
+      const bool two = q + 32 < hot.count;
+      const uint32_t e1 = two ? hot.slots[q + 32] : e0;
+      const int g0 = (int)(e0 >> 5) * (int)blockDim.x + wbase + (int)(e0 & 31);
+      const int g1 = (int)(e1 >> 5) * (int)blockDim.x + wbase + (int)(e1 & 31);
+      Granule<TIn> a0, a1;
+      a0.load_any(row, V, n_full, g0);
+      if (two) a1.load_any(row, V, n_full, g1);
+      granule_masked_sum<TIn>(a0, g0, a, st.tau, st.m, sc);
+      if (two) granule_masked_sum<TIn>(a1, g1, a, st.tau, st.m, sc);
     }
   } else {
-    for (int i = 0; i < n_steps; ++i) {
-      if (chunk_max[i * blockDim.x + tid] >= st.tau) {
-        Chunk<TIn, kUnroll> c;
-        c.load(row, V, n_full, i * per_sweep, tid);
-        chunk_masked_sum<TIn, kUnroll>(c, i * per_sweep, tid, a, va, st.tau, st.m, sc);
+    for (int i = 0; i < n_slots; ++i) {
+      if (bf16_bits_to_float(bound[i * blockDim.x + tid]) >= st.tau) {
+        const int g = i * (int)blockDim.x + tid;
+        Granule<TIn> gr;
+        gr.load_any(row, V, n_full, g);
+        granule_masked_sum<TIn>(gr, g, a, st.tau, st.m, sc);
       }
     }
   }
@@ -197,100 +340,71 @@ __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int a, dou
   return st;
 }
 
-// Gradient entries of one chunk (Prop. 5.4, set fixed), stored to the row.
-template <typename TIn, typename TGrad, int kUnroll>
-__device__ __forceinline__ void chunk_grad(const Chunk<TIn, kUnroll> &c, TGrad *grow, int V,
-                                           int n_full, int n_vec, int vb, int tid, int a, int va,
-                                           float tau, float m, float coef, float g_a) {
-  constexpr int kPerVec = Storage<TIn>::kPerVec;
-#pragma unroll
-  for (int u = 0; u < kUnroll; ++u) {
-    const int v = vb + u * (int)blockDim.x + tid;
-    if (v >= n_vec) continue;
-    float x[kPerVec], out[kPerVec];
-    c.get(u, x);
-    const int ja = v == va ? a - va * kPerVec : -1;
-#pragma unroll
-    for (int j = 0; j < kPerVec; ++j) {
-      out[j] = x[j] >= tau ? coef * ex2((x[j] - m) * kLog2e) : 0.f;
-      if (j == ja) out[j] = g_a;
-    }
-    if (v < n_full) {
-      store_grads<TGrad, kPerVec>(grow + (size_t)v * kPerVec, out);
-    } else {
-#pragma unroll
-      for (int j = 0; j < kPerVec; ++j) {
-        const long long k = (long long)v * kPerVec + j;
-        if (k < V) grow[k] = Storage<TGrad>::narrow(out[j]);
-      }
-    }
-  }
-}
-
-// Sweep 3: gradient of g * ln pi^mp(a) over the row.  Chunks without a safe
+// Sweep 3: gradient of g * ln pi^mp(a) over the row.  Granules without a safe
 // token are written as zeros without being read.
-template <typename TIn, typename TGrad, int kUnroll>
+template <typename TIn, typename TGrad, int kStage>
 __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int a,
-                                         const SideStats &st, float g, const float *chunk_max,
+                                         const SideStats &st, float g, const uint16_t *bound,
                                          const HotList &hot) {
-  constexpr int kPerVec = Storage<TIn>::kPerVec;
-  const int n_full = V / kPerVec;
-  const int n_vec = (V + kPerVec - 1) / kPerVec;
-  const int per_sweep = kUnroll * (int)blockDim.x;
-  const int n_steps = (n_vec + per_sweep - 1) / per_sweep;
+  constexpr int kElems = Granule<TIn>::kElems;
+  const int n_full = V / kElems;
+  const int n_gran = (V + kElems - 1) / kElems;
+  const int per_step = kStage * (int)blockDim.x;
+  const int n_slots = ((n_gran + per_step - 1) / per_step) * kStage;
   const int tid = threadIdx.x;
   const float s_safe = st.s_x + st.e_a;
   // a pruned or missing sampled token has weight zero: the row is all zeros
   const bool live = st.member;
   const float coef = live ? -g / s_safe : 0.f;
   const float g_a = live ? g * (st.s_x / s_safe) : 0.f;
-  const int va = live ? a / kPerVec : -1;
+  const int a_live = live ? a : -1;
   const bool listed = live && hot.fits();
   const float tau = live ? st.tau : -kNegInf;  // +inf: nothing passes
 
-  for (int i = 0; i < n_steps; ++i) {
-    const int vb = i * per_sweep;
-    if (chunk_max[i * blockDim.x + tid] >= tau) {
+  for (int i = 0; i < n_slots; ++i) {
+    const int gi = i * (int)blockDim.x + tid;
+    if (gi >= n_gran) break;
+    if (bf16_bits_to_float(bound[i * blockDim.x + tid]) >= tau) {
       if (!listed) {
-        Chunk<TIn, kUnroll> c;
-        c.load(row, V, n_full, vb, tid);
-        chunk_grad<TIn, TGrad, kUnroll>(c, grow, V, n_full, n_vec, vb, tid, a, va, tau, st.m, coef,
-                                        g_a);
+        Granule<TIn> gr;
+        gr.load_any(row, V, n_full, gi);
+        granule_grad<TIn, TGrad>(gr, grow, V, n_full, gi, a_live, tau, st.m, coef, g_a);
       }
-      continue;
-    }
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const int v = vb + u * (int)blockDim.x + tid;
-      if (v < n_full) {
-        store_zeros<TGrad, kPerVec>(grow + (size_t)v * kPerVec);
-      } else if (v < n_vec) {
-        for (int j = 0; j < kPerVec; ++j) {
-          const long long k = (long long)v * kPerVec + j;
-          if (k < V) grow[k] = Storage<TGrad>::narrow(0.f);
-        }
+    } else if (gi < n_full) {
+      store_zero_granule<TGrad, kElems>(grow + (size_t)gi * kElems);
+    } else {
+      for (int j = 0; j < kElems; ++j) {
+        const long long k = (long long)gi * kElems + j;
+        if (k < V) grow[k] = Storage<TGrad>::narrow(0.f);
       }
     }
   }
   if (listed) {
-    const int wbase = tid & ~31;
-    for (int q = tid & 31; q < hot.count; q += 32) {
-      const uint32_t e = hot.slots[q];
-      const int vb = (int)(e >> 5) * per_sweep, owner = wbase + (int)(e & 31);
-      Chunk<TIn, kUnroll> c;
-      c.load(row, V, n_full, vb, owner);
-      chunk_grad<TIn, TGrad, kUnroll>(c, grow, V, n_full, n_vec, vb, owner, a, va, tau, st.m, coef,
-                                      g_a);
+    const int wbase = tid & ~31, lane = tid & 31;
+    for (int q = lane; q < hot.count; q += 64) {
+      const uint32_t e0 = hot.slots[q];
+      const bool two = q + 32 < hot.count;
+      const uint32_t e1 = two ? hot.slots[q + 32] : e0;
+      const int g0 = (int)(e0 >> 5) * (int)blockDim.x + wbase + (int)(e0 & 31);
+      const int g1 = (int)(e1 >> 5) * (int)blockDim.x + wbase + (int)(e1 & 31);
+      Granule<TIn> a0, a1;
+      a0.load_any(row, V, n_full, g0);
+      if (two) a1.load_any(row, V, n_full, g1);
+      granule_grad<TIn, TGrad>(a0, grow, V, n_full, g0, a_live, tau, st.m, coef, g_a);
+      if (two) granule_grad<TIn, TGrad>(a1, grow, V, n_full, g1, a_live, tau, st.m, coef, g_a);
     }
   }
 }
 
-template <typename TIn, typename TGrad, int kUnroll>
+// Shared-memory layout of the row kernel, in 4-byte words.
+__host__ __device__ inline int smem_words_fixed(int threads) { return 96 + (threads / 32) * kHotCap; }
+
+template <typename TIn, typename TGrad, int kStage>
 __global__ void __launch_bounds__(512, 2) dvp_row_kernel(const RowParams p) {
   extern __shared__ __align__(16) float smem[];
-  float *scratch = smem;  // 64 floats for the block reductions
-  uint32_t *hot_smem = reinterpret_cast<uint32_t *>(smem + 64);  // kHotCap per warp
-  float *chunk_max = smem + 64 + (blockDim.x >> 5) * kHotCap;    // one float per (step, thread)
+  float *scratch = smem;  // 96 floats for the block reductions
+  uint32_t *hot_smem = reinterpret_cast<uint32_t *>(smem + 96);  // kHotCap per warp
+  uint16_t *bound = reinterpret_cast<uint16_t *>(smem + smem_words_fixed(blockDim.x));
 
   const long long t = blockIdx.x;
   const long long id = p.ids ? load_id(p.ids, p.id_is_i32, t) : -1;
@@ -302,21 +416,21 @@ __global__ void __launch_bounds__(512, 2) dvp_row_kernel(const RowParams p) {
   uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * ((p.V + 31) / 32) : nullptr;
   HotList hot;
   const SideStats st =
-      row_stats<TIn, kUnroll>(trow, V, a, p.log_rho, chunk_max, scratch, hot_smem, hot, mask_t);
+      row_stats<TIn, kStage>(trow, V, a, p.log_rho, bound, scratch, hot_smem, hot, mask_t);
 
   if (p.grad) {
     const float g = p.upstream[t];
-    row_grad<TIn, TGrad, kUnroll>(trow, reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad, V, a, st,
-                                  g, chunk_max, hot);
+    row_grad<TIn, TGrad, kStage>(trow, reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad, V, a, st,
+                                 g, bound, hot);
   }
 
   SideStats si;
   if (p.infer) {
-    __syncthreads();  // chunk_max and the hot lists are reused for the second matrix
+    __syncthreads();  // the bounds and the hot lists are reused for the second matrix
     const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
     uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
     HotList hot_i;
-    si = row_stats<TIn, kUnroll>(irow, V, a, p.log_rho, chunk_max, scratch, hot_smem, hot_i, mask_i);
+    si = row_stats<TIn, kStage>(irow, V, a, p.log_rho, bound, scratch, hot_smem, hot_i, mask_i);
   }
 
   if (threadIdx.x == 0) {
@@ -336,7 +450,7 @@ __global__ void __launch_bounds__(512, 2) dvp_row_kernel(const RowParams p) {
 
 // ---- scalar kernel: any alignment, any row length ---------------------------
 // Three plain sweeps per matrix with element-wise loads; used when a row does
-// not start on a 16-byte boundary or is too long for the chunk summary.
+// not start on a 32-byte boundary or is too long for the granule bounds.
 
 template <typename TIn>
 __device__ __forceinline__ SideStats row_stats_scalar(const TIn *row, long long V, long long a,
@@ -351,7 +465,7 @@ __device__ __forceinline__ SideStats row_stats_scalar(const TIn *row, long long 
   const MaxSum all = block_reduce_maxsum(acc, scratch);
   SideStats st;
   st.m = all.m;
-  st.s = all.s;
+  st.lse = (double)all.m + (double)logf(all.s);
   st.tau = threshold_f32(all.m, log_rho);
   const bool has_a = a >= 0 && a < V;
   st.z_a = has_a ? Storage<TIn>::widen(row[a]) : 0.f;
@@ -433,9 +547,8 @@ __global__ void dvp_row_kernel_scalar(const RowParams p) {
 
 // ---- stand-alone backward: a streaming map from saved row statistics ---------
 
-template <typename TIn, typename TGrad, int kUnroll, bool kVector>
+template <typename TIn, typename TGrad, int kStage, bool kVector>
 __global__ void dvp_backward_kernel(const BackwardParams p) {
-  constexpr int kPerVec = Storage<TIn>::kPerVec;
   const long long t = blockIdx.x;
   const TIn *row = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
   TGrad *grow = reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad;
@@ -453,33 +566,23 @@ __global__ void dvp_backward_kernel(const BackwardParams p) {
     g_a = g * comp;
   }
   if constexpr (kVector) {
+    constexpr int kElems = Granule<TIn>::kElems;
     const int V = (int)p.V;
-    const int n_full = V / kPerVec;
-    const int n_vec = (V + kPerVec - 1) / kPerVec;
-    const int per_sweep = kUnroll * (int)blockDim.x;
-    const int va = live ? (int)(a / kPerVec) : -1;
-    for (int vb = 0; vb < n_vec; vb += per_sweep) {
-      Chunk<TIn, kUnroll> c;
-      c.load(row, V, n_full, vb, threadIdx.x);
+    const int n_full = V / kElems;
+    const int n_gran = (V + kElems - 1) / kElems;
+    const int per_step = kStage * (int)blockDim.x;
+    for (int gb = 0; gb < n_gran; gb += per_step) {
+      Granule<TIn> gr[kStage];
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        const int v = vb + u * (int)blockDim.x + threadIdx.x;
-        if (v >= n_vec) continue;
-        float x[kPerVec], out[kPerVec];
-        c.get(u, x);
-        const int ja = v == va ? (int)a - va * kPerVec : -1;
+      for (int u = 0; u < kStage; ++u) {
+        const int gi = gb + u * (int)blockDim.x + threadIdx.x;
+        if (gi < n_gran) gr[u].load_any(row, V, n_full, gi);
+      }
 #pragma unroll
-        for (int j = 0; j < kPerVec; ++j) {
-          out[j] = x[j] >= tau ? coef * ex2((x[j] - m) * kLog2e) : 0.f;
-          if (j == ja) out[j] = g_a;
-        }
-        if (v < n_full) {
-          store_grads<TGrad, kPerVec>(grow + (size_t)v * kPerVec, out);
-        } else {
-#pragma unroll
-          for (int j = 0; j < kPerVec; ++j)
-            if ((long long)v * kPerVec + j < V) grow[(long long)v * kPerVec + j] = Storage<TGrad>::narrow(out[j]);
-        }
+      for (int u = 0; u < kStage; ++u) {
+        const int gi = gb + u * (int)blockDim.x + threadIdx.x;
+        if (gi < n_gran)
+          granule_grad<TIn, TGrad>(gr[u], grow, V, n_full, gi, (int)a, tau, m, coef, g_a);
       }
     }
   } else {
@@ -494,13 +597,13 @@ __global__ void dvp_backward_kernel(const BackwardParams p) {
 
 // ---- host-side launchers ------------------------------------------------------
 
-static bool aligned16(const void *base, long long ld, size_t elem) {
-  return base == nullptr || (((uintptr_t)base % 16 == 0) && ((ld * (long long)elem) % 16 == 0));
+static bool aligned32(const void *base, long long ld, size_t elem) {
+  return base == nullptr || (((uintptr_t)base % 32 == 0) && ((ld * (long long)elem) % 32 == 0));
 }
 
-template <typename TIn, typename TGrad, int kUnroll>
+template <typename TIn, typename TGrad, int kStage>
 static cudaError_t launch_rows_vec(const RowParams &p, int threads, size_t smem, cudaStream_t s) {
-  auto k = dvp_row_kernel<TIn, TGrad, kUnroll>;
+  auto k = dvp_row_kernel<TIn, TGrad, kStage>;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -511,28 +614,23 @@ static cudaError_t launch_rows_vec(const RowParams &p, int threads, size_t smem,
 
 template <typename TIn, typename TGrad>
 static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s) {
-  constexpr int kPerVec = Storage<TIn>::kPerVec;
-  int threads = hint & 0xffff, unroll = (hint >> 16) & 0xff;
+  constexpr int kElems = Granule<TIn>::kElems;
+  int threads = hint & 0xffff, stage = (hint >> 16) & 0xff;
   if (threads == 0) threads = 256;
-  if (unroll == 0) unroll = 4;
-  const bool vec_ok = aligned16(p.train, p.ld_train, sizeof(TIn)) &&
-                      aligned16(p.infer, p.ld_infer, sizeof(TIn)) &&
-                      aligned16(p.grad, p.ld_grad, sizeof(TGrad));
-  const long long n_vec = (p.V + kPerVec - 1) / kPerVec;
+  if (stage == 0) stage = 2;
+  const bool vec_ok = aligned32(p.train, p.ld_train, sizeof(TIn)) &&
+                      aligned32(p.infer, p.ld_infer, sizeof(TIn)) &&
+                      aligned32(p.grad, p.ld_grad, sizeof(TGrad));
+  const long long n_gran = (p.V + kElems - 1) / kElems;
   // shrink the block for short rows so that threads are not idle
-  while (threads > 64 && (long long)threads * unroll / 2 >= n_vec) threads /= 2;
-  auto smem_for = [&](int u) {
-    const long long per = (long long)u * threads;
-    return (size_t)(64 + (threads / 32) * kHotCap + ((n_vec + per - 1) / per) * threads) * sizeof(float);
-  };
-  const size_t smem_cap = 200 * 1024;
-  if (vec_ok) {
-    if (unroll < 4) unroll = 4;
-    while (unroll < 8 && smem_for(unroll) > 72 * 1024) unroll *= 2;
-    if (smem_for(unroll) <= smem_cap) {
-      if (unroll <= 4) return launch_rows_vec<TIn, TGrad, 4>(p, threads, smem_for(4), s);
-      return launch_rows_vec<TIn, TGrad, 8>(p, threads, smem_for(8), s);
-    }
+  while (threads > 64 && (long long)threads * stage / 2 >= n_gran) threads /= 2;
+  const long long per = (long long)stage * threads;
+  const size_t smem = (size_t)smem_words_fixed(threads) * 4 +
+                      (size_t)((n_gran + per - 1) / per) * per * sizeof(uint16_t);
+  if (vec_ok && smem <= 200 * 1024) {
+    if (stage <= 1) return launch_rows_vec<TIn, TGrad, 1>(p, threads, smem, s);
+    if (stage <= 2) return launch_rows_vec<TIn, TGrad, 2>(p, threads, smem, s);
+    return launch_rows_vec<TIn, TGrad, 4>(p, threads, smem, s);
   }
   dvp_row_kernel_scalar<TIn, TGrad><<<(unsigned)p.T, 512, 0, s>>>(p);
   return cudaGetLastError();
@@ -561,9 +659,9 @@ static cudaError_t launch_bwd(const BackwardParams &p, uint32_t hint, cudaStream
   int threads = hint & 0xffff;
   if (threads == 0) threads = 256;
   const bool vec_ok =
-      aligned16(p.train, p.ld_train, sizeof(TIn)) && aligned16(p.grad, p.ld_grad, sizeof(TGrad));
+      aligned32(p.train, p.ld_train, sizeof(TIn)) && aligned32(p.grad, p.ld_grad, sizeof(TGrad));
   if (vec_ok)
-    dvp_backward_kernel<TIn, TGrad, 4, true><<<(unsigned)p.T, threads, 0, s>>>(p);
+    dvp_backward_kernel<TIn, TGrad, 2, true><<<(unsigned)p.T, threads, 0, s>>>(p);
   else
     dvp_backward_kernel<TIn, TGrad, 1, false><<<(unsigned)p.T, threads, 0, s>>>(p);
   return cudaGetLastError();
