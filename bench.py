@@ -42,7 +42,7 @@ NCU_TRAFFIC = {
 def _kernel_digest() -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2512_23087_b200", "csrc")
-    for name in ("dvp_common.cuh", "dvp_rows.cu"):
+    for name in ("dvp_common.cuh", "dvp_rows_impl.cuh"):
         h.update(open(os.path.join(csrc, name), "rb").read())
     return h.hexdigest()[:16]
 

@@ -1,688 +1,31 @@
-// Row kernels of Dynamic Vocabulary Pruning for sm_100a.
-//
-// One thread block owns one token row.  The row is streamed from HBM once
-// (sweep 1) in 32-byte granules, one DRAM sector per lane and load, two
-// pipeline stages deep.  While it streams, every thread keeps an online
-// log-sum-exp of what it has seen and leaves in shared memory an upper bound
-// (bfloat16, rounded up) of the maximum of each granule it loaded.  Once the
-// row maximum, hence the threshold of Def. 5.1, is known, only granules whose
-// bound reaches the threshold can hold safe tokens: sweep 2 (masked sum and
-// count, Def. 5.2) and sweep 3 (gradient, Prop. 5.4) revisit just those, and
-// sweep 3 writes zeros for all the others without reading anything.  With a
-// sparse safe set a row costs one HBM read per logit matrix and one HBM write
-// of the gradient; with a dense safe set the same code degrades to three
-// sweeps, still correct.
+// Dispatch of the row kernels on the logits type; the kernels themselves are in
+// dvp_rows_impl.cuh and are compiled once per type in dvp_rows_{f32,bf16,f16}.cu.
 #include "dvp_common.cuh"
 
 namespace dvp {
 
-template <typename T>
-struct Pair;
-template <>
-struct Pair<__nv_bfloat16> {
-  using type = __nv_bfloat162;
-};
-template <>
-struct Pair<__half> {
-  using type = __half2;
-};
-
-// ---- a 32-byte granule of a row, kept packed as loaded ------------------------
-
-template <typename TIn>
-struct Granule {
-  static constexpr int kElems = 32 / (int)sizeof(TIn);
-  uint32_t w[8];
-
-  __device__ __forceinline__ void load(const TIn *p) { ld_stream32(p, w); }
-
-  // Granule `g` of a row of V elements; elements past V read as -inf.
-  __device__ __forceinline__ void load_any(const TIn *row, int V, int n_full, int g) {
-    if (g < n_full) {
-      load(row + (size_t)g * kElems);
-    } else {
-      __align__(16) TIn tmp[kElems];
-#pragma unroll
-      for (int j = 0; j < kElems; ++j) {
-        const long long k = (long long)g * kElems + j;
-        tmp[j] = k < V ? row[k] : Storage<TIn>::narrow(kNegInf);
-      }
-#pragma unroll
-      for (int i = 0; i < 8; ++i) w[i] = reinterpret_cast<const uint32_t *>(tmp)[i];
-    }
-  }
-
-  __device__ __forceinline__ void get(float *x) const {
-    constexpr int kHalf = kElems / 2;
-    Storage<TIn>::unpack(make_uint4(w[0], w[1], w[2], w[3]), x);
-    Storage<TIn>::unpack(make_uint4(w[4], w[5], w[6], w[7]), x + kHalf);
-  }
-
-  __device__ __forceinline__ float max() const {
-    if constexpr (sizeof(TIn) == 4) {
-      float m = __uint_as_float(w[0]);
-#pragma unroll
-      for (int i = 1; i < 8; ++i) m = fmaxf(m, __uint_as_float(w[i]));
-      return m;
-    } else {
-      // packed two-at-a-time maxima, then the two halves of the last pair
-      using T2 = typename Pair<TIn>::type;
-      T2 p[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) p[i] = *reinterpret_cast<const T2 *>(&w[i]);
-#pragma unroll
-      for (int s = 4; s > 0; s >>= 1)
-#pragma unroll
-        for (int i = 0; i < s; ++i) p[i] = __hmax2(p[i], p[i + s]);
-      return fmaxf(Storage<TIn>::widen(p[0].x), Storage<TIn>::widen(p[0].y));
-    }
-  }
-};
-
-// Upper bound of a float as a bfloat16 bit pattern (round toward +inf).
-__device__ __forceinline__ uint16_t bf16_bits_round_up(float v) {
-  const uint32_t b = __float_as_uint(v);
-  // positive: bump the magnitude unless the low half is zero; negative: truncate
-  return (uint16_t)(((b & 0x80000000u) ? b : b + 0xffffu) >> 16);
-}
-__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
-  return __uint_as_float((uint32_t)b << 16);
-}
-
-template <typename TGrad, int kElems>
-__device__ __forceinline__ void store_granule(TGrad *dst, const float *out) {
-  constexpr int kBytes = kElems * (int)sizeof(TGrad);
-  if constexpr (sizeof(TGrad) == 4) {
-#pragma unroll
-    for (int i = 0; i < kElems; i += 8) {
-      uint32_t w[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) w[j] = __float_as_uint(out[i + j]);
-      st_stream32(dst + i, w);
-    }
-  } else {
-    uint32_t w[kElems / 2];
-#pragma unroll
-    for (int i = 0; i < kElems / 2; ++i) {
-      TGrad lo = Storage<TGrad>::narrow(out[2 * i]), hi = Storage<TGrad>::narrow(out[2 * i + 1]);
-      w[i] = (uint32_t) * reinterpret_cast<uint16_t *>(&lo) |
-             ((uint32_t) * reinterpret_cast<uint16_t *>(&hi) << 16);
-    }
-    if constexpr (kBytes == 32) {
-      uint32_t v[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) v[i] = w[i];
-      st_stream32(dst, v);
-    } else {
-      static_assert(kBytes == 16, "granule of 8 floats stored as 8 halves");
-      st_stream16(dst, make_uint4(w[0], w[1], w[2], w[3]));
-    }
-  }
-}
-
-template <typename TGrad, int kElems>
-__device__ __forceinline__ void store_zero_granule(TGrad *dst) {
-  constexpr int kBytes = kElems * (int)sizeof(TGrad);
-  const uint32_t z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  if constexpr (kBytes == 64) {
-    st_stream32(dst, z);
-    st_stream32(reinterpret_cast<char *>(dst) + 32, z);
-  } else if constexpr (kBytes == 32) {
-    st_stream32(dst, z);
-  } else {
-    st_stream16(dst, make_uint4(0, 0, 0, 0));
-  }
-}
-
-// ---- granules that can hold a safe token ----------------------------------------
-// Per warp, in the order (slot, lane): entry = ordinal of the granule among the
-// warp's granules.  A warp whose hot granules do not fit (a dense safe set)
-// walks all of its granules instead, which is then the efficient thing to do.
-constexpr int kHotCap = 256;
-
-struct HotList {
-  uint32_t *slots;
-  int count;  // granules at or above the threshold (may exceed kHotCap)
-  __device__ __forceinline__ bool fits() const { return count <= kHotCap; }
-};
-
-__device__ __forceinline__ HotList build_hot_list(const uint16_t *bound, int n_slots, float tau,
-                                                  uint32_t *hot_smem) {
-  const int lane = threadIdx.x & 31;
-  HotList h;
-  h.slots = hot_smem + (threadIdx.x >> 5) * kHotCap;
-  h.count = 0;
-  for (int i = 0; i < n_slots; ++i) {
-    const bool f = bf16_bits_to_float(bound[i * blockDim.x + threadIdx.x]) >= tau;
-    const unsigned b = __ballot_sync(0xffffffffu, f);
-    if (f) {
-      const int pos = h.count + __popc(b & ((1u << lane) - 1u));
-      if (pos < kHotCap) h.slots[pos] = (uint32_t)(i * 32 + lane);
-    }
-    h.count += __popc(b);
-  }
-  __syncwarp();
-  return h;
-}
-
-// Contribution of one granule to the masked sum and the count (Def. 5.2).
-template <typename TIn>
-__device__ __forceinline__ void granule_masked_sum(const Granule<TIn> &gr, int g, int a, float tau,
-                                                   float m, SumCount &sc) {
-  constexpr int kElems = Granule<TIn>::kElems;
-  float x[kElems];
-  gr.get(x);
-  // the sampled token is left out so that 1 - pi^mp(a) has no cancellation
-  const int ja = a - g * kElems;  // in [0, kElems) only inside the owner granule
-#pragma unroll
-  for (int j = 0; j < kElems; ++j) {
-    if (x[j] >= tau) {
-      ++sc.n;
-      if (j != ja) sc.s += ex2((x[j] - m) * kLog2e);
-    }
-  }
-}
-
-// Gradient entries of one granule (Prop. 5.4, set fixed), stored to the row.
-template <typename TIn, typename TGrad>
-__device__ __forceinline__ void granule_grad(const Granule<TIn> &gr, TGrad *grow, int V, int n_full,
-                                             int g, int a, float tau, float m, float coef,
-                                             float g_a) {
-  constexpr int kElems = Granule<TIn>::kElems;
-  float x[kElems], out[kElems];
-  gr.get(x);
-  const int ja = a - g * kElems;
-#pragma unroll
-  for (int j = 0; j < kElems; ++j) {
-    out[j] = x[j] >= tau ? coef * ex2((x[j] - m) * kLog2e) : 0.f;
-    if (j == ja) out[j] = g_a;
-  }
-  if (g < n_full) {
-    store_granule<TGrad, kElems>(grow + (size_t)g * kElems, out);
-  } else {
-#pragma unroll
-    for (int j = 0; j < kElems; ++j) {
-      const long long k = (long long)g * kElems + j;
-      if (k < V) grow[k] = Storage<TGrad>::narrow(out[j]);
-    }
-  }
-}
-
-// One pipeline stage of sweep 1: kStage granules of this thread.
-template <typename TIn, int kStage>
-struct Stage {
-  Granule<TIn> g[kStage];
-  __device__ __forceinline__ void load(const TIn *row, int V, int n_full, int step) {
-    const int g0 = step * kStage * (int)blockDim.x + threadIdx.x;
-    if ((step + 1) * kStage * (int)blockDim.x <= n_full) {
-#pragma unroll
-      for (int u = 0; u < kStage; ++u)
-        g[u].load(row + (size_t)(g0 + u * (int)blockDim.x) * Granule<TIn>::kElems);
-    } else {
-#pragma unroll
-      for (int u = 0; u < kStage; ++u) g[u].load_any(row, V, n_full, g0 + u * (int)blockDim.x);
-    }
-  }
-};
-
-template <typename TIn, int kStage>
-__device__ __forceinline__ void absorb_stage(const Stage<TIn, kStage> &st, int step, LogSum &acc,
-                                             uint16_t *bound) {
-  constexpr int kElems = Granule<TIn>::kElems;
-  float cm = kNegInf;
-#pragma unroll
-  for (int u = 0; u < kStage; ++u) {
-    const float gm = st.g[u].max();
-    bound[(step * kStage + u) * blockDim.x + threadIdx.x] = bf16_bits_round_up(gm);
-    cm = fmaxf(cm, gm);
-  }
-  if (cm > kNegInf) {
-    if (cm > acc.m) {
-      const float cn = cm * kLog2e;
-      acc.s *= ex2(acc.c - cn);  // acc.c = -inf at the start: the factor is 0
-      acc.m = cm;
-      acc.c = cn;
-    }
-    const float neg_c = -acc.c;
-    float part = 0.f;
-#pragma unroll
-    for (int u = 0; u < kStage; ++u) {
-      float x[kElems];
-      st.g[u].get(x);
-#pragma unroll
-      for (int j = 0; j < kElems; ++j) part += ex2(fmaf(x[j], kLog2e, neg_c));
-    }
-    acc.s += part;
-  }
-}
-
-// Sweeps 1 and 2 over one row: statistics of one side.
-template <typename TIn, int kStage>
-__device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int a, double log_rho,
-                                               uint16_t *bound, float *scratch, uint32_t *hot_smem,
-                                               HotList &hot, uint32_t *mask_row) {
-  constexpr int kElems = Granule<TIn>::kElems;
-  const int n_full = V / kElems;
-  const int n_gran = (V + kElems - 1) / kElems;
-  const int per_step = kStage * (int)blockDim.x;
-  const int n_steps = (n_gran + per_step - 1) / per_step;
-  const int tid = threadIdx.x;
-
-  // ---- sweep 1, two stages in flight
-  LogSum acc = {kNegInf, kNegInf, 0.f};
-  {
-    Stage<TIn, kStage> s0, s1;
-    s0.load(row, V, n_full, 0);
-    int step = 0;
-    for (; step + 1 < n_steps; step += 2) {
-      s1.load(row, V, n_full, step + 1);
-      absorb_stage<TIn, kStage>(s0, step, acc, bound);
-      if (step + 2 < n_steps) s0.load(row, V, n_full, step + 2);
-      absorb_stage<TIn, kStage>(s1, step + 1, acc, bound);
-    }
-    if (step < n_steps) absorb_stage<TIn, kStage>(s0, step, acc, bound);
-  }
-  const LogSum all = block_reduce_logsum(acc, scratch);
-
-  SideStats st;
-  st.m = all.m;
-  st.lse = lse_from_logsum(all);
-  st.tau = threshold_f32(all.m, log_rho);
-  const bool has_a = a >= 0 && a < V;
-  st.z_a = has_a ? Storage<TIn>::widen(row[a]) : 0.f;
-  st.member = has_a && st.z_a >= st.tau;
-  st.e_a = st.member ? ex2((st.z_a - st.m) * kLog2e) : 0.f;
-
-  // ---- sweep 2: only granules that can hold a safe token
-  SumCount sc = {0.f, 0};
-  const int n_slots = n_steps * kStage;  // granules per thread
-  hot = build_hot_list(bound, n_slots, st.tau, hot_smem);
-  if (hot.fits()) {
-    const int wbase = tid & ~31, lane = tid & 31;
-    for (int q = lane; q < hot.count; q += 64) {
-      const uint32_t e0 = hot.slots[q];
-      const bool two = q + 32 < hot.count;
-      const uint32_t e1 = two ? hot.slots[q + 32] : e0;
-      const int g0 = (int)(e0 >> 5) * (int)blockDim.x + wbase + (int)(e0 & 31);
-      const int g1 = (int)(e1 >> 5) * (int)blockDim.x + wbase + (int)(e1 & 31);
-      Granule<TIn> a0, a1;
-      a0.load_any(row, V, n_full, g0);
-      if (two) a1.load_any(row, V, n_full, g1);
-      granule_masked_sum<TIn>(a0, g0, a, st.tau, st.m, sc);
-      if (two) granule_masked_sum<TIn>(a1, g1, a, st.tau, st.m, sc);
-    }
-  } else {
-    for (int i = 0; i < n_slots; ++i) {
-      if (bf16_bits_to_float(bound[i * blockDim.x + tid]) >= st.tau) {
-        const int g = i * (int)blockDim.x + tid;
-        Granule<TIn> gr;
-        gr.load_any(row, V, n_full, g);
-        granule_masked_sum<TIn>(gr, g, a, st.tau, st.m, sc);
-      }
-    }
-  }
-  const SumCount tot = block_reduce_sumcount(sc, scratch);
-  st.s_x = tot.s;
-  st.n = tot.n;
-
-  // ---- optional packed membership mask (diagnostic output, plain loads)
-  if (mask_row) {
-    const int n_words = (V + 31) / 32;
-    for (int w = tid; w < n_words; w += blockDim.x) {
-      uint32_t bits = 0;
-      for (int b = 0; b < 32; ++b) {
-        const long long k = (long long)w * 32 + b;
-        if (k < V && Storage<TIn>::widen(row[k]) >= st.tau) bits |= 1u << b;
-      }
-      mask_row[w] = bits;
-    }
-  }
-  return st;
-}
-
-// Sweep 3: gradient of g * ln pi^mp(a) over the row.  Granules without a safe
-// token are written as zeros without being read.
-template <typename TIn, typename TGrad, int kStage>
-__device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int a,
-                                         const SideStats &st, float g, const uint16_t *bound,
-                                         const HotList &hot) {
-  constexpr int kElems = Granule<TIn>::kElems;
-  const int n_full = V / kElems;
-  const int n_gran = (V + kElems - 1) / kElems;
-  const int per_step = kStage * (int)blockDim.x;
-  const int n_slots = ((n_gran + per_step - 1) / per_step) * kStage;
-  const int tid = threadIdx.x;
-  const float s_safe = st.s_x + st.e_a;
-  // a pruned or missing sampled token has weight zero: the row is all zeros
-  const bool live = st.member;
-  const float coef = live ? -g / s_safe : 0.f;
-  const float g_a = live ? g * (st.s_x / s_safe) : 0.f;
-  const int a_live = live ? a : -1;
-  const bool listed = live && hot.fits();
-  const float tau = live ? st.tau : -kNegInf;  // +inf: nothing passes
-
-  for (int i = 0; i < n_slots; ++i) {
-    const int gi = i * (int)blockDim.x + tid;
-    if (gi >= n_gran) break;
-    if (bf16_bits_to_float(bound[i * blockDim.x + tid]) >= tau) {
-      if (!listed) {
-        Granule<TIn> gr;
-        gr.load_any(row, V, n_full, gi);
-        granule_grad<TIn, TGrad>(gr, grow, V, n_full, gi, a_live, tau, st.m, coef, g_a);
-      }
-    } else if (gi < n_full) {
-      store_zero_granule<TGrad, kElems>(grow + (size_t)gi * kElems);
-    } else {
-      for (int j = 0; j < kElems; ++j) {
-        const long long k = (long long)gi * kElems + j;
-        if (k < V) grow[k] = Storage<TGrad>::narrow(0.f);
-      }
-    }
-  }
-  if (listed) {
-    const int wbase = tid & ~31, lane = tid & 31;
-    for (int q = lane; q < hot.count; q += 64) {
-      const uint32_t e0 = hot.slots[q];
-      const bool two = q + 32 < hot.count;
-      const uint32_t e1 = two ? hot.slots[q + 32] : e0;
-      const int g0 = (int)(e0 >> 5) * (int)blockDim.x + wbase + (int)(e0 & 31);
-      const int g1 = (int)(e1 >> 5) * (int)blockDim.x + wbase + (int)(e1 & 31);
-      Granule<TIn> a0, a1;
-      a0.load_any(row, V, n_full, g0);
-      if (two) a1.load_any(row, V, n_full, g1);
-      granule_grad<TIn, TGrad>(a0, grow, V, n_full, g0, a_live, tau, st.m, coef, g_a);
-      if (two) granule_grad<TIn, TGrad>(a1, grow, V, n_full, g1, a_live, tau, st.m, coef, g_a);
-    }
-  }
-}
-
-// Shared-memory layout of the row kernel, in 4-byte words.
-__host__ __device__ inline int smem_words_fixed(int threads) { return 96 + (threads / 32) * kHotCap; }
-
-template <typename TIn, typename TGrad, int kStage>
-__global__ void __launch_bounds__(512, 2) dvp_row_kernel(const RowParams p) {
-  extern __shared__ __align__(16) float smem[];
-  float *scratch = smem;  // 96 floats for the block reductions
-  uint32_t *hot_smem = reinterpret_cast<uint32_t *>(smem + 96);  // kHotCap per warp
-  uint16_t *bound = reinterpret_cast<uint16_t *>(smem + smem_words_fixed(blockDim.x));
-
-  const long long t = blockIdx.x;
-  const long long id = p.ids ? load_id(p.ids, p.id_is_i32, t) : -1;
-  const bool has_id = id >= 0, bad_id = id >= p.V;
-  const int a = (has_id && !bad_id) ? (int)id : -1;
-  const int V = (int)p.V;
-
-  const TIn *trow = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
-  uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * ((p.V + 31) / 32) : nullptr;
-  HotList hot;
-  const SideStats st =
-      row_stats<TIn, kStage>(trow, V, a, p.log_rho, bound, scratch, hot_smem, hot, mask_t);
-
-  if (p.grad) {
-    const float g = p.upstream[t];
-    row_grad<TIn, TGrad, kStage>(trow, reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad, V, a, st,
-                                 g, bound, hot);
-  }
-
-  SideStats si;
-  if (p.infer) {
-    __syncthreads();  // the bounds and the hot lists are reused for the second matrix
-    const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
-    uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
-    HotList hot_i;
-    si = row_stats<TIn, kStage>(irow, V, a, p.log_rho, bound, scratch, hot_smem, hot_i, mask_i);
-  }
-
-  if (threadIdx.x == 0) {
-    const float lt = finish_side(p.out_t, t, st, has_id, bad_id);
-    uint8_t flags = (uint8_t)((st.member ? DVP_FLAG_IN_TRAIN : 0) | (has_id ? 0 : DVP_FLAG_NO_ID) |
-                              (bad_id ? DVP_FLAG_BAD_ID : 0));
-    if (p.infer) {
-      const float li = finish_side(p.out_i, t, si, has_id, bad_id);
-      if (si.member) flags |= DVP_FLAG_IN_INFER;
-      if (p.log_ratio)
-        p.log_ratio[t] = (has_id && !bad_id) ? log_ratio_of(st.member, si.member, lt, li)
-                                             : __int_as_float(0x7fc00000);
-    }
-    if (p.flags) p.flags[t] = flags;
-  }
-}
-
-// ---- scalar kernel: any alignment, any row length ---------------------------
-// Three plain sweeps per matrix with element-wise loads; used when a row does
-// not start on a 32-byte boundary or is too long for the granule bounds.
-
-template <typename TIn>
-__device__ __forceinline__ SideStats row_stats_scalar(const TIn *row, long long V, long long a,
-                                                      double log_rho, float *scratch,
-                                                      uint32_t *mask_row) {
-  float m = kNegInf;
-  for (long long k = threadIdx.x; k < V; k += blockDim.x) m = fmaxf(m, Storage<TIn>::widen(row[k]));
-  MaxSum acc = {m, 0.f};
-  if (m > kNegInf)
-    for (long long k = threadIdx.x; k < V; k += blockDim.x)
-      acc.s += ex2((Storage<TIn>::widen(row[k]) - m) * kLog2e);
-  const MaxSum all = block_reduce_maxsum(acc, scratch);
-  SideStats st;
-  st.m = all.m;
-  st.lse = (double)all.m + (double)logf(all.s);
-  st.tau = threshold_f32(all.m, log_rho);
-  const bool has_a = a >= 0 && a < V;
-  st.z_a = has_a ? Storage<TIn>::widen(row[a]) : 0.f;
-  st.member = has_a && st.z_a >= st.tau;
-  st.e_a = st.member ? ex2((st.z_a - st.m) * kLog2e) : 0.f;
-  SumCount sc = {0.f, 0};
-  for (long long k = threadIdx.x; k < V; k += blockDim.x) {
-    const float z = Storage<TIn>::widen(row[k]);
-    if (z >= st.tau) {
-      ++sc.n;
-      if (k != a) sc.s += ex2((z - st.m) * kLog2e);
-    }
-  }
-  const SumCount tot = block_reduce_sumcount(sc, scratch);
-  st.s_x = tot.s;
-  st.n = tot.n;
-  if (mask_row) {
-    const long long n_words = (V + 31) / 32;
-    for (long long w = threadIdx.x; w < n_words; w += blockDim.x) {
-      uint32_t bits = 0;
-      for (int b = 0; b < 32; ++b) {
-        const long long k = w * 32 + b;
-        if (k < V && Storage<TIn>::widen(row[k]) >= st.tau) bits |= 1u << b;
-      }
-      mask_row[w] = bits;
-    }
-  }
-  return st;
-}
-
-template <typename TIn, typename TGrad>
-__global__ void dvp_row_kernel_scalar(const RowParams p) {
-  __shared__ float scratch[64];
-  const long long t = blockIdx.x;
-  const long long id = p.ids ? load_id(p.ids, p.id_is_i32, t) : -1;
-  const bool has_id = id >= 0, bad_id = id >= p.V;
-  const long long a = (has_id && !bad_id) ? id : -1;
-
-  const TIn *trow = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
-  uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * ((p.V + 31) / 32) : nullptr;
-  const SideStats st = row_stats_scalar<TIn>(trow, p.V, a, p.log_rho, scratch, mask_t);
-
-  if (p.grad) {
-    TGrad *grow = reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad;
-    const float g = p.upstream[t];
-    const float s_safe = st.s_x + st.e_a;
-    const bool live = st.member;
-    const float coef = live ? -g / s_safe : 0.f;
-    const float g_a = live ? g * (st.s_x / s_safe) : 0.f;
-    for (long long k = threadIdx.x; k < p.V; k += blockDim.x) {
-      const float z = Storage<TIn>::widen(trow[k]);
-      float out = (live && z >= st.tau) ? coef * ex2((z - st.m) * kLog2e) : 0.f;
-      if (live && k == a) out = g_a;
-      grow[k] = Storage<TGrad>::narrow(out);
-    }
-  }
-
-  SideStats si;
-  if (p.infer) {
-    const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
-    uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
-    si = row_stats_scalar<TIn>(irow, p.V, a, p.log_rho, scratch, mask_i);
-  }
-
-  if (threadIdx.x == 0) {
-    const float lt = finish_side(p.out_t, t, st, has_id, bad_id);
-    uint8_t flags = (uint8_t)((st.member ? DVP_FLAG_IN_TRAIN : 0) | (has_id ? 0 : DVP_FLAG_NO_ID) |
-                              (bad_id ? DVP_FLAG_BAD_ID : 0));
-    if (p.infer) {
-      const float li = finish_side(p.out_i, t, si, has_id, bad_id);
-      if (si.member) flags |= DVP_FLAG_IN_INFER;
-      if (p.log_ratio)
-        p.log_ratio[t] = (has_id && !bad_id) ? log_ratio_of(st.member, si.member, lt, li)
-                                             : __int_as_float(0x7fc00000);
-    }
-    if (p.flags) p.flags[t] = flags;
-  }
-}
-
-// ---- stand-alone backward: a streaming map from saved row statistics ---------
-
-template <typename TIn, typename TGrad, int kStage, bool kVector>
-__global__ void dvp_backward_kernel(const BackwardParams p) {
-  const long long t = blockIdx.x;
-  const TIn *row = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
-  TGrad *grow = reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad;
-  const long long id = load_id(p.ids, p.id_is_i32, t);
-  const bool live = (p.flags[t] & DVP_FLAG_IN_TRAIN) && id >= 0 && id < p.V;
-  const long long a = live ? id : -1;
-  const float g = p.upstream[t], m = p.max_t[t];
-  const float tau = live ? threshold_f32(m, p.log_rho) : -kNegInf;
-  // e^{z - lse_safe} = e^{z - m} e^{m - lse_safe}; the second factor is 1 / s_safe
-  const float coef = live ? -g * ex2((m - p.lse_safe_t[t]) * kLog2e) : 0.f;
-  float g_a = 0.f;
-  if (live) {
-    const float comp = p.comp_mp_t ? p.comp_mp_t[t]
-                                   : -expm1f(Storage<TIn>::widen(row[a]) - p.lse_safe_t[t]);
-    g_a = g * comp;
-  }
-  if constexpr (kVector) {
-    constexpr int kElems = Granule<TIn>::kElems;
-    const int V = (int)p.V;
-    const int n_full = V / kElems;
-    const int n_gran = (V + kElems - 1) / kElems;
-    const int per_step = kStage * (int)blockDim.x;
-    for (int gb = 0; gb < n_gran; gb += per_step) {
-      Granule<TIn> gr[kStage];
-#pragma unroll
-      for (int u = 0; u < kStage; ++u) {
-        const int gi = gb + u * (int)blockDim.x + threadIdx.x;
-        if (gi < n_gran) gr[u].load_any(row, V, n_full, gi);
-      }
-#pragma unroll
-      for (int u = 0; u < kStage; ++u) {
-        const int gi = gb + u * (int)blockDim.x + threadIdx.x;
-        if (gi < n_gran)
-          granule_grad<TIn, TGrad>(gr[u], grow, V, n_full, gi, (int)a, tau, m, coef, g_a);
-      }
-    }
-  } else {
-    for (long long k = threadIdx.x; k < p.V; k += blockDim.x) {
-      const float z = Storage<TIn>::widen(row[k]);
-      float out = z >= tau ? coef * ex2((z - m) * kLog2e) : 0.f;
-      if (k == a) out = g_a;
-      grow[k] = Storage<TGrad>::narrow(out);
-    }
-  }
-}
-
-// ---- host-side launchers ------------------------------------------------------
-
-static bool aligned32(const void *base, long long ld, size_t elem) {
-  return base == nullptr || (((uintptr_t)base % 32 == 0) && ((ld * (long long)elem) % 32 == 0));
-}
-
-template <typename TIn, typename TGrad, int kStage>
-static cudaError_t launch_rows_vec(const RowParams &p, int threads, size_t smem, cudaStream_t s) {
-  auto k = dvp_row_kernel<TIn, TGrad, kStage>;
-  if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-  }
-  k<<<(unsigned)p.T, threads, smem, s>>>(p);
-  return cudaGetLastError();
-}
-
-template <typename TIn, typename TGrad>
-static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s) {
-  constexpr int kElems = Granule<TIn>::kElems;
-  int threads = hint & 0xffff, stage = (hint >> 16) & 0xff;
-  if (threads == 0) threads = 256;
-  if (stage == 0) stage = 2;
-  const bool vec_ok = aligned32(p.train, p.ld_train, sizeof(TIn)) &&
-                      aligned32(p.infer, p.ld_infer, sizeof(TIn)) &&
-                      aligned32(p.grad, p.ld_grad, sizeof(TGrad));
-  const long long n_gran = (p.V + kElems - 1) / kElems;
-  // shrink the block for short rows so that threads are not idle
-  while (threads > 64 && (long long)threads * stage / 2 >= n_gran) threads /= 2;
-  const long long per = (long long)stage * threads;
-  const size_t smem = (size_t)smem_words_fixed(threads) * 4 +
-                      (size_t)((n_gran + per - 1) / per) * per * sizeof(uint16_t);
-  if (vec_ok && smem <= 200 * 1024) {
-    if (stage <= 1) return launch_rows_vec<TIn, TGrad, 1>(p, threads, smem, s);
-    if (stage <= 2) return launch_rows_vec<TIn, TGrad, 2>(p, threads, smem, s);
-    return launch_rows_vec<TIn, TGrad, 4>(p, threads, smem, s);
-  }
-  dvp_row_kernel_scalar<TIn, TGrad><<<(unsigned)p.T, 512, 0, s>>>(p);
-  return cudaGetLastError();
-}
-
-template <typename TIn>
-static cudaError_t launch_rows_g(const RowParams &p, int grad_dtype, uint32_t hint, cudaStream_t s) {
-  switch (grad_dtype) {
-    case DVP_F32: return launch_rows<TIn, float>(p, hint, s);
-    case DVP_BF16: return launch_rows<TIn, __nv_bfloat16>(p, hint, s);
-    default: return launch_rows<TIn, __half>(p, hint, s);
-  }
-}
+cudaError_t launch_row_kernels_f32(const RowParams &, int, uint32_t, cudaStream_t);
+cudaError_t launch_row_kernels_bf16(const RowParams &, int, uint32_t, cudaStream_t);
+cudaError_t launch_row_kernels_f16(const RowParams &, int, uint32_t, cudaStream_t);
+cudaError_t launch_backward_kernel_f32(const BackwardParams &, int, uint32_t, cudaStream_t);
+cudaError_t launch_backward_kernel_bf16(const BackwardParams &, int, uint32_t, cudaStream_t);
+cudaError_t launch_backward_kernel_f16(const BackwardParams &, int, uint32_t, cudaStream_t);
 
 cudaError_t launch_row_kernels(const RowParams &p, int logits_dtype, int grad_dtype, uint32_t hint,
                                cudaStream_t s) {
   switch (logits_dtype) {
-    case DVP_F32: return launch_rows_g<float>(p, grad_dtype, hint, s);
-    case DVP_BF16: return launch_rows_g<__nv_bfloat16>(p, grad_dtype, hint, s);
-    default: return launch_rows_g<__half>(p, grad_dtype, hint, s);
-  }
-}
-
-template <typename TIn, typename TGrad>
-static cudaError_t launch_bwd(const BackwardParams &p, uint32_t hint, cudaStream_t s) {
-  int threads = hint & 0xffff;
-  if (threads == 0) threads = 256;
-  const bool vec_ok =
-      aligned32(p.train, p.ld_train, sizeof(TIn)) && aligned32(p.grad, p.ld_grad, sizeof(TGrad));
-  if (vec_ok)
-    dvp_backward_kernel<TIn, TGrad, 2, true><<<(unsigned)p.T, threads, 0, s>>>(p);
-  else
-    dvp_backward_kernel<TIn, TGrad, 1, false><<<(unsigned)p.T, threads, 0, s>>>(p);
-  return cudaGetLastError();
-}
-
-template <typename TIn>
-static cudaError_t launch_bwd_g(const BackwardParams &p, int grad_dtype, uint32_t hint,
-                                cudaStream_t s) {
-  switch (grad_dtype) {
-    case DVP_F32: return launch_bwd<TIn, float>(p, hint, s);
-    case DVP_BF16: return launch_bwd<TIn, __nv_bfloat16>(p, hint, s);
-    default: return launch_bwd<TIn, __half>(p, hint, s);
+    case DVP_F32: return launch_row_kernels_f32(p, grad_dtype, hint, s);
+    case DVP_BF16: return launch_row_kernels_bf16(p, grad_dtype, hint, s);
+    default: return launch_row_kernels_f16(p, grad_dtype, hint, s);
   }
 }
 
 cudaError_t launch_backward_kernel(const BackwardParams &p, int logits_dtype, int grad_dtype,
                                    uint32_t hint, cudaStream_t s) {
   switch (logits_dtype) {
-    case DVP_F32: return launch_bwd_g<float>(p, grad_dtype, hint, s);
-    case DVP_BF16: return launch_bwd_g<__nv_bfloat16>(p, grad_dtype, hint, s);
-    default: return launch_bwd_g<__half>(p, grad_dtype, hint, s);
+    case DVP_F32: return launch_backward_kernel_f32(p, grad_dtype, hint, s);
+    case DVP_BF16: return launch_backward_kernel_bf16(p, grad_dtype, hint, s);
+    default: return launch_backward_kernel_f16(p, grad_dtype, hint, s);
   }
 }
 
