@@ -33,9 +33,12 @@ UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes per launch of the row kernel (dram__bytes_read.sum + dram__bytes_write.sum
-# from one ncu capture), keyed by workload; valid only for the kernel sources whose
-# digest is recorded with it, scaled by rows when the capture used fewer rows.
+# from one ncu capture of `bench.py --rows T ...`), keyed by (workload, rho); valid only for
+# the kernel sources whose digest is recorded with it, scaled by rows to the full batch.
 NCU_TRAFFIC = {
+    ("c2_bf16_fwdbwd", 1e-4): {"digest": "f616e3106fa1d8d0", "T": 2048, "bytes": 1.638192e9 + 0.605876e9},
+    ("c2_bf16_fwdbwd", 1e-3): {"digest": "f616e3106fa1d8d0", "T": 2048, "bytes": 1.351455e9 + 0.608828e9},
+    ("c3_f32_heavy", 1e-4): {"digest": "f616e3106fa1d8d0", "T": 1024, "bytes": 2.148637e9 + 1.072640e9},
 }
 
 
@@ -317,9 +320,9 @@ def run_ours(args):
     alg_bytes = (2 * elem + (grad_elem if w.backward else 0)) * T * V
     achieved = alg_bytes / (ms * 1e-3 / args.steps) / 1e9
     traffic = None
-    rec = NCU_TRAFFIC.get(w.name)
-    if rec and rec.get("digest") == _kernel_digest() and rec.get("rho") == rho:
-        traffic = rec["bytes"] * (T / rec["T"])
+    rec = NCU_TRAFFIC.get((w.name, rho))
+    if rec and rec["digest"] == _kernel_digest():
+        traffic = rec["bytes"] * (T / rec["T"])      # rows are independent: traffic grows with T
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -216,7 +216,7 @@ def test_results_do_not_depend_on_launch_shape_and_are_reproducible():
     assert torch.equal(base.grad_train, again.grad_train)
     want = parity.run_oracle(batch.train, batch.infer, batch.ids, 1e-4, batch.upstream)
     for threads in (64, 128, 512):
-        for unroll in (1, 2, 4):
+        for unroll in (1, 2):
             res = _forward(batch, 1e-4, True, launch_hint=threads | (unroll << 16))
             torch.cuda.synchronize()
             assert torch.equal(res.train.count, base.train.count)
