@@ -182,18 +182,25 @@ int dvp_backward(const dvp_backward_args *args);
  *   hidden        device [T, ld_hidden] bf16
  *   w_vocab       device [V, ld_w] bf16
  *   infer_logits  device [T, ld_infer] bf16 (what the inference engine
- *                 computed for the same parameters), or NULL
+ *                 computed for the same parameters), or NULL (then `infer`
+ *                 outputs and log_ratio must be NULL)
  *   d_hidden      device [T, ld_dh] float32, overwritten
  *   d_w           device [V, ld_dw] float32; overwritten, or added to when
  *                 accumulate_dw != 0
  *   workspace     device, 256-byte aligned, at least
- *                 dvp_workspace_bytes(DVP_ENTRY_FUSED_LMHEAD, args) bytes
- *   panel_rows    0 = library default; otherwise a multiple of 128
+ *                 dvp_workspace_bytes(DVP_ENTRY_FUSED_LMHEAD, args) bytes.
+ *                 Its first 32-bit word is a status: 0 after a run in which
+ *                 every tensor-core kernel finished, non-zero if one gave up
+ *                 waiting (results are then invalid).
+ *   panel_rows    0 = library default (at most 4096); otherwise a multiple of 128
  *
- * H must be a multiple of 64 and rows of hidden, w_vocab must start on
- * 16-byte boundaries (DVP_ERR_UNSUPPORTED otherwise).  Membership is decided
- * on the fp32-accumulated logits, so a token whose logit sits within rounding
- * distance of the threshold may fall on either side.
+ * ld_hidden, ld_w, ld_dh, ld_dw must be multiples of 8 and hidden, w_vocab
+ * 16-byte, d_hidden, d_w 32-byte aligned (DVP_ERR_UNSUPPORTED otherwise).
+ * Membership is decided on the fp32-accumulated logits, so a token whose logit
+ * sits within rounding distance of the threshold may fall on either side of
+ * the exact-arithmetic decision.  The gradient panel is held in float16 times
+ * a power of two taken from max |upstream|: entries more than about 2^-28
+ * below max |upstream| lose relative accuracy.
  */
 typedef struct {
   uint32_t struct_size;
@@ -220,6 +227,21 @@ typedef struct {
 } dvp_fused_args;
 
 int dvp_fused_lmhead_forward_backward(const dvp_fused_args *args);
+
+/*
+ * dvp_gemm_tn -- the tensor-core contraction the fused entry point is built on,
+ * exposed for reuse and testing: C[m, n] (+)= alpha * A[m, k] * B[n, k]^T with A
+ * and B both bf16 or both f16 (dtype), row-major with k contiguous, C float32
+ * row-major, fp32 accumulation.  The paper has no counterpart; it is the
+ * "hidden x W_vocab" product of the LM head and its two transposes.
+ *   a, b, c   device; lda, ldb, ldc multiples of 8; a, b 16-byte, c 32-byte aligned
+ *   status    device int32, written non-zero if a kernel gave up waiting
+ * Errors: DVP_ERR_INVALID_ARG (null pointers, negative sizes),
+ * DVP_ERR_UNSUPPORTED (dtype, alignment), DVP_ERR_CUDA.
+ */
+int dvp_gemm_tn(const void *a, int64_t lda, const void *b, int64_t ldb, float *c, int64_t ldc,
+                int64_t m, int64_t n, int64_t k, int32_t dtype, float alpha, int32_t accumulate,
+                int32_t *status, void *stream);
 
 /*
  * Bytes of device workspace the entry point needs for `args` (a pointer to

@@ -22,7 +22,7 @@ DVP_ID_I64, DVP_ID_I32 = 0, 1
 DVP_FLAG_IN_TRAIN, DVP_FLAG_IN_INFER, DVP_FLAG_NO_ID, DVP_FLAG_BAD_ID = 1, 2, 64, 128
 DVP_ENTRY_FORWARD, DVP_ENTRY_BACKWARD, DVP_ENTRY_FUSED_LMHEAD = 0, 1, 2
 
-EXPORTS = ("dvp_forward", "dvp_backward", "dvp_fused_lmhead_forward_backward",
+EXPORTS = ("dvp_forward", "dvp_backward", "dvp_fused_lmhead_forward_backward", "dvp_gemm_tn",
            "dvp_workspace_bytes", "dvp_status_string", "dvp_version")
 
 _DTYPES = {torch.float32: DVP_F32, torch.bfloat16: DVP_BF16, torch.float16: DVP_F16}
@@ -141,6 +141,11 @@ def load_library() -> ctypes.CDLL:
         lib.dvp_backward.restype = ctypes.c_int
         lib.dvp_fused_lmhead_forward_backward.argtypes = [ctypes.POINTER(FusedArgs)]
         lib.dvp_fused_lmhead_forward_backward.restype = ctypes.c_int
+        lib.dvp_gemm_tn.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64,
+                                    ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                                    ctypes.c_int64, ctypes.c_int32, ctypes.c_float, ctypes.c_int32,
+                                    ctypes.c_void_p, ctypes.c_void_p]
+        lib.dvp_gemm_tn.restype = ctypes.c_int
         lib.dvp_workspace_bytes.argtypes = [ctypes.c_int, ctypes.c_void_p]
         lib.dvp_workspace_bytes.restype = ctypes.c_size_t
         lib.dvp_status_string.argtypes = [ctypes.c_int]
@@ -283,6 +288,28 @@ def dvp_backward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, upst
     if st != DVP_OK:
         raise DvpError(st, "dvp_backward")
     return grad_train
+
+
+def dvp_gemm_tn(a: torch.Tensor, b: torch.Tensor, *, alpha: float = 1.0, out: torch.Tensor | None = None,
+                accumulate: bool = False, stream=None):
+    """``out (+)= alpha * a @ b.T`` on the tensor cores; a [m, k] and b [n, k] are
+    both bf16 or both f16 with k contiguous, out is float32.  Returns (out, status)
+    where status is a device int32 that is non-zero if the kernel gave up waiting."""
+    lib = load_library()
+    _check_matrix("a", a)
+    _check_matrix("b", b)
+    if a.dtype != b.dtype or a.dtype not in (torch.bfloat16, torch.float16):
+        raise TypeError("a and b must both be bfloat16 or both float16")
+    m, k = a.shape
+    n = b.shape[0]
+    if out is None:
+        out = torch.empty(m, n, dtype=torch.float32, device=a.device)
+    status = torch.zeros(1, dtype=torch.int32, device=a.device)
+    st = lib.dvp_gemm_tn(_ptr(a), a.stride(0), _ptr(b), b.stride(0), _ptr(out), out.stride(0), m, n, k,
+                         _DTYPES[a.dtype], float(alpha), int(accumulate), _ptr(status), _stream(stream))
+    if st != DVP_OK:
+        raise DvpError(st, "dvp_gemm_tn")
+    return out, status
 
 
 def dvp_workspace_bytes(entry_point: int, args: ctypes.Structure) -> int:

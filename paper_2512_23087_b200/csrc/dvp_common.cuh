@@ -288,6 +288,7 @@ __device__ __forceinline__ SumCount block_reduce_sumcount(SumCount v, float *scr
 struct RowParams {
   const void *train, *infer, *ids;
   const float *upstream;
+  const float *grad_scale;  // optional device scalar multiplied into every upstream gradient
   void *grad;
   long long T, V, ld_train, ld_infer, ld_grad;
   double log_rho;  // ln(rho); -inf for rho = 0

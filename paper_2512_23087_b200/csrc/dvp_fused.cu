@@ -1,17 +1,279 @@
-// Fused LM-head entry point (placeholder until the tensor-core path lands).
+// Fused LM-head entry point: z = hidden x W_vocab^T on the tensor cores, the
+// row computation of dvp_forward on panels of those logits, and the chain rule
+// through the head (d_hidden = G W, d_w = G^T hidden) as two more contractions.
+//
+// The [T, V] training logits are never stored: a panel of `panel_rows` tokens
+// lives in the workspace as fp32 logits, is turned into the gradient panel G by
+// the ordinary row kernel, and is consumed by the two gradient contractions
+// before the next panel overwrites it.
+//
+// G is held in float16 (11-bit significand; bfloat16's 8 bits would miss the
+// 1e-3 gradient tolerance by themselves) times a power of two chosen from
+// max |upstream| so that the panel uses float16's normal range; the inverse
+// power of two is applied in the epilogues of the gradient contractions.
+// tcgen05 kind::f16 needs both operands of one type, so W^T and hidden^T are
+// converted to float16 copies once per call (exact for bfloat16 values in
+// float16's normal range).
+#include <cmath>
+
 #include "dvp_common.cuh"
+#include "dvp_gemm.cuh"
+
+namespace dvp {
+
+// out[c, r] = convert(in[r, c]) for a row-major [R, C] input.
+template <typename TIn, typename TOut>
+__global__ void transpose_convert_kernel(const TIn *in, long long ld_in, TOut *out, long long ld_out,
+                                         int R, int C) {
+  __shared__ float tile[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+    const int r = r0 + j, c = c0 + threadIdx.x;
+    tile[j][threadIdx.x] = (r < R && c < C) ? Storage<TIn>::widen(in[(long long)r * ld_in + c]) : 0.f;
+  }
+  __syncthreads();
+  for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+    const int c = c0 + j, r = r0 + threadIdx.x;
+    if (c < C && r < R) out[(long long)c * ld_out + r] = Storage<TOut>::narrow(tile[threadIdx.x][j]);
+  }
+}
+
+struct FusedScalars {
+  int status;       // non-zero when a tensor-core kernel gave up waiting
+  float scale;      // power of two applied to the gradient panel
+  float inv_scale;  // its inverse
+};
+
+// scale = 2^(14 - x) with max|g| < 2^x, so that |scale * G| < 2^14.
+__global__ void grad_scale_kernel(const float *upstream, long long T, FusedScalars *out) {
+  __shared__ float red[32];
+  float m = 0.f;
+  for (long long t = threadIdx.x; t < T; t += blockDim.x) {
+    const float v = fabsf(upstream[t]);
+    if (v < __int_as_float(0x7f800000)) m = fmaxf(m, v);
+  }
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) m = fmaxf(m, red[w]);
+    int x = 0;
+    if (m > 0.f) frexpf(m, &x);
+    int e = 14 - x;
+    e = e > 60 ? 60 : (e < -60 ? -60 : e);
+    out->status = 0;
+    out->scale = ldexpf(1.f, e);
+    out->inv_scale = ldexpf(1.f, -e);
+  }
+}
+
+// Merge the two sides: flags and the per-token log-ratio.
+__global__ void combine_sides_kernel(long long T, const float *lp_t, const float *lp_i,
+                                     const uint8_t *flags_i, uint8_t *flags, float *log_ratio) {
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= T) return;
+  const uint8_t ft = flags[t];
+  const bool in_t = ft & DVP_FLAG_IN_TRAIN, in_i = flags_i[t] & DVP_FLAG_IN_TRAIN;
+  flags[t] = (uint8_t)(ft | (in_i ? DVP_FLAG_IN_INFER : 0));
+  if (log_ratio)
+    log_ratio[t] = (ft & (DVP_FLAG_NO_ID | DVP_FLAG_BAD_ID)) ? __int_as_float(0x7fc00000)
+                                                             : log_ratio_of(in_t, in_i, lp_t[t], lp_i[t]);
+}
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct FusedLayout {
+  long long Vp, Tp, panel;
+  size_t off_scalars, off_lpt, off_lpi, off_fli, off_flt, off_wt, off_ht, off_z, off_g, off_gt, total;
+};
+
+bool fused_layout(const dvp_fused_args *a, FusedLayout *L) {
+  if (a->T < 0 || a->H < 1 || a->V < 1) return false;
+  long long panel = a->panel_rows;
+  if (panel == 0) {
+    panel = (a->T + 127) / 128 * 128;
+    if (panel > 4096) panel = 4096;
+    if (panel < 128) panel = 128;
+  }
+  if (panel % 128 != 0 || panel < 128) return false;
+  L->panel = panel;
+  L->Vp = (a->V + 15) / 16 * 16;
+  L->Tp = (a->T + 7) / 8 * 8;
+  if (L->Tp == 0) L->Tp = 8;
+  size_t o = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = o;
+    o = align_up(o + bytes, 256);
+    return at;
+  };
+  L->off_scalars = take(sizeof(FusedScalars));
+  L->off_lpt = take((size_t)a->T * 4);
+  L->off_lpi = take((size_t)a->T * 4);
+  L->off_fli = take((size_t)a->T);
+  L->off_flt = take((size_t)a->T);
+  L->off_wt = take((size_t)a->H * L->Vp * 2);
+  L->off_ht = take((size_t)a->H * L->Tp * 2);
+  L->off_z = take((size_t)panel * L->Vp * 4);
+  L->off_g = take((size_t)panel * L->Vp * 2);
+  L->off_gt = take((size_t)a->V * panel * 2);
+  L->total = o;
+  return true;
+}
+
+dvp_side_out offset_side(const dvp_side_out &o, long long r0, long long words) {
+  dvp_side_out r = o;
+  if (r.max) r.max += r0;
+  if (r.lse) r.lse += r0;
+  if (r.lse_safe) r.lse_safe += r0;
+  if (r.logp) r.logp += r0;
+  if (r.logp_mp) r.logp_mp += r0;
+  if (r.comp_mp) r.comp_mp += r0;
+  if (r.count) r.count += r0;
+  if (r.mask) r.mask += r0 * words;
+  return r;
+}
+
+}  // namespace
+}  // namespace dvp
 
 extern "C" {
 
-int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
-  if (!a || a->struct_size != sizeof(dvp_fused_args)) return DVP_ERR_INVALID_ARG;
-  return DVP_ERR_UNSUPPORTED;
+size_t dvp_workspace_bytes(int entry_point, const void *args) {
+  if (entry_point != DVP_ENTRY_FUSED_LMHEAD || !args) return 0;
+  const dvp_fused_args *a = static_cast<const dvp_fused_args *>(args);
+  if (a->struct_size != sizeof(dvp_fused_args)) return 0;
+  dvp::FusedLayout L;
+  return dvp::fused_layout(a, &L) ? L.total : 0;
 }
 
-size_t dvp_workspace_bytes(int entry_point, const void *args) {
-  (void)entry_point;
-  (void)args;
-  return 0;
+int dvp_gemm_tn(const void *a, int64_t lda, const void *b, int64_t ldb, float *c, int64_t ldc, int64_t m,
+                int64_t n, int64_t k, int32_t dtype, float alpha, int32_t accumulate, int32_t *status,
+                void *stream) {
+  if (!a || !b || !c || !status || m < 0 || n < 0 || k < 0) return DVP_ERR_INVALID_ARG;
+  if (m > 0x7fffffffLL || n > 0x7fffffffLL || k > 0x7fffffffLL) return DVP_ERR_UNSUPPORTED;
+  if (dtype != DVP_BF16 && dtype != DVP_F16) return DVP_ERR_UNSUPPORTED;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return DVP_ERR_CUDA;
+  const cudaError_t e =
+      dvp::gemm::launch_gemm_tn(a, lda, b, ldb, c, ldc, (int)m, (int)n, (int)k, dtype == DVP_BF16, alpha,
+                                nullptr, accumulate != 0, status, sms, static_cast<cudaStream_t>(stream));
+  if (e == cudaErrorInvalidValue) return DVP_ERR_UNSUPPORTED;
+  return e == cudaSuccess ? DVP_OK : DVP_ERR_CUDA;
+}
+
+int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
+  using namespace dvp;
+  if (!a || a->struct_size != sizeof(dvp_fused_args)) return DVP_ERR_INVALID_ARG;
+  if (a->id_dtype != DVP_ID_I64 && a->id_dtype != DVP_ID_I32) return DVP_ERR_UNSUPPORTED;
+  if (a->T < 0 || a->T > 0x7fffffffLL || a->H < 1 || a->V < 1) return DVP_ERR_INVALID_ARG;
+  if (a->V > 0x7fffff00LL || a->H > 0x7fffff00LL) return DVP_ERR_UNSUPPORTED;
+  if (!(a->rho >= 0.0 && a->rho <= 1.0)) return DVP_ERR_INVALID_ARG;
+  FusedLayout L;
+  if (!fused_layout(a, &L)) return DVP_ERR_INVALID_ARG;
+  if (a->T == 0) return DVP_OK;
+  if (!a->hidden || !a->w_vocab || !a->ids || !a->upstream || !a->d_hidden || !a->d_w)
+    return DVP_ERR_INVALID_ARG;
+  if (a->ld_hidden < a->H || a->ld_w < a->H || a->ld_dh < a->H || a->ld_dw < a->H)
+    return DVP_ERR_INVALID_ARG;
+  if (a->infer_logits && a->ld_infer < a->V) return DVP_ERR_INVALID_ARG;
+  if (!a->infer_logits && a->log_ratio) return DVP_ERR_INVALID_ARG;
+  if (a->ld_hidden % 8 || a->ld_w % 8 || a->ld_dh % 8 || a->ld_dw % 8 ||
+      (uintptr_t)a->hidden % 16 || (uintptr_t)a->w_vocab % 16 || (uintptr_t)a->d_hidden % 32 ||
+      (uintptr_t)a->d_w % 32)
+    return DVP_ERR_UNSUPPORTED;
+  if (!a->workspace || (uintptr_t)a->workspace % 256 || a->workspace_bytes < L.total)
+    return DVP_ERR_WORKSPACE;
+
+  cudaStream_t s = static_cast<cudaStream_t>(a->stream);
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return DVP_ERR_CUDA;
+
+  char *ws = static_cast<char *>(a->workspace);
+  FusedScalars *sc = reinterpret_cast<FusedScalars *>(ws + L.off_scalars);
+  float *lpt = a->train.logp_mp ? a->train.logp_mp : reinterpret_cast<float *>(ws + L.off_lpt);
+  float *lpi = a->infer.logp_mp ? a->infer.logp_mp : reinterpret_cast<float *>(ws + L.off_lpi);
+  uint8_t *fli = reinterpret_cast<uint8_t *>(ws + L.off_fli);
+  uint8_t *flt = a->flags ? a->flags : reinterpret_cast<uint8_t *>(ws + L.off_flt);
+  __half *wt16 = reinterpret_cast<__half *>(ws + L.off_wt);   // [H, Vp]: W^T
+  __half *ht16 = reinterpret_cast<__half *>(ws + L.off_ht);   // [H, Tp]: hidden^T
+  float *z = reinterpret_cast<float *>(ws + L.off_z);         // [panel, Vp] logits
+  __half *g16 = reinterpret_cast<__half *>(ws + L.off_g);     // [panel, Vp] scaled gradient
+  __half *gt16 = reinterpret_cast<__half *>(ws + L.off_gt);   // [V, panel]: its transpose
+  const __nv_bfloat16 *hidden = static_cast<const __nv_bfloat16 *>(a->hidden);
+  const __nv_bfloat16 *w = static_cast<const __nv_bfloat16 *>(a->w_vocab);
+  const int T = (int)a->T, H = (int)a->H, V = (int)a->V;
+  const long long id_bytes = a->id_dtype == DVP_ID_I32 ? 4 : 8;
+  const long long mask_words = (a->V + 31) / 32;
+
+  grad_scale_kernel<<<1, 1024, 0, s>>>(a->upstream, a->T, sc);
+  const dim3 tb(32, 8);
+  transpose_convert_kernel<__nv_bfloat16, __half>
+      <<<dim3((H + 31) / 32, (V + 31) / 32), tb, 0, s>>>(w, a->ld_w, wt16, L.Vp, V, H);
+  transpose_convert_kernel<__nv_bfloat16, __half>
+      <<<dim3((H + 31) / 32, (T + 31) / 32), tb, 0, s>>>(hidden, a->ld_hidden, ht16, L.Tp, T, H);
+  if (cudaGetLastError() != cudaSuccess) return DVP_ERR_CUDA;
+
+  const double log_rho = a->rho > 0.0 ? std::log(a->rho) : -HUGE_VAL;
+  int panel_index = 0;
+  for (long long r0 = 0; r0 < a->T; r0 += L.panel, ++panel_index) {
+    const int rows = (int)((a->T - r0 < L.panel) ? a->T - r0 : L.panel);
+    // logits of the panel: z = hidden[r0 : r0 + rows] x W^T (bf16 operands, fp32 accumulate)
+    cudaError_t e = gemm::launch_gemm_tn(hidden + r0 * a->ld_hidden, a->ld_hidden, w, a->ld_w, z, L.Vp,
+                                         rows, V, H, true, 1.f, nullptr, false, &sc->status, sms, s);
+    if (e != cudaSuccess) return e == cudaErrorInvalidValue ? DVP_ERR_UNSUPPORTED : DVP_ERR_CUDA;
+    // rows of the panel: statistics and G = scale * dLoss/dz in float16
+    RowParams p{};
+    p.train = z;
+    p.ids = static_cast<const char *>(a->ids) + r0 * id_bytes;
+    p.upstream = a->upstream + r0;
+    p.grad_scale = &sc->scale;
+    p.grad = g16;
+    p.T = rows;
+    p.V = a->V;
+    p.ld_train = L.Vp;
+    p.ld_grad = L.Vp;
+    p.log_rho = log_rho;
+    p.id_is_i32 = a->id_dtype == DVP_ID_I32;
+    p.out_t = offset_side(a->train, r0, mask_words);
+    p.out_t.logp_mp = lpt + r0;
+    p.flags = flt + r0;
+    if (launch_row_kernels(p, DVP_F32, DVP_F16, 0, s) != cudaSuccess) return DVP_ERR_CUDA;
+    transpose_convert_kernel<__half, __half>
+        <<<dim3((V + 31) / 32, (rows + 31) / 32), tb, 0, s>>>(g16, L.Vp, gt16, L.panel, rows, V);
+    // d_hidden[r0 : r0 + rows] = G x W / scale
+    e = gemm::launch_gemm_tn(g16, L.Vp, wt16, L.Vp, a->d_hidden + r0 * a->ld_dh, a->ld_dh, rows, H, V,
+                             false, 1.f, &sc->inv_scale, false, &sc->status, sms, s);
+    if (e != cudaSuccess) return e == cudaErrorInvalidValue ? DVP_ERR_UNSUPPORTED : DVP_ERR_CUDA;
+    // d_w (+)= G^T x hidden[r0 : r0 + rows] / scale
+    e = gemm::launch_gemm_tn(gt16, L.panel, ht16 + r0, L.Tp, a->d_w, a->ld_dw, V, H, rows, false, 1.f,
+                             &sc->inv_scale, panel_index > 0 || a->accumulate_dw != 0, &sc->status, sms,
+                             s);
+    if (e != cudaSuccess) return e == cudaErrorInvalidValue ? DVP_ERR_UNSUPPORTED : DVP_ERR_CUDA;
+  }
+
+  if (a->infer_logits) {
+    RowParams p{};
+    p.train = a->infer_logits;
+    p.ids = a->ids;
+    p.T = a->T;
+    p.V = a->V;
+    p.ld_train = a->ld_infer;
+    p.log_rho = log_rho;
+    p.id_is_i32 = a->id_dtype == DVP_ID_I32;
+    p.out_t = a->infer;
+    p.out_t.logp_mp = lpi;
+    p.flags = fli;
+    if (launch_row_kernels(p, DVP_BF16, DVP_BF16, 0, s) != cudaSuccess) return DVP_ERR_CUDA;
+    combine_sides_kernel<<<(unsigned)((a->T + 255) / 256), 256, 0, s>>>(a->T, lpt, lpi, fli, flt,
+                                                                        a->log_ratio);
+  }
+  return cudaGetLastError() == cudaSuccess ? DVP_OK : DVP_ERR_CUDA;
 }
 
 }  // extern "C"

@@ -1,0 +1,377 @@
+// Tensor-core contraction C[M,N] (+)= alpha * A[M,K] * B[N,K]^T for sm_100a.
+//
+// A and B are 16-bit (both bf16 or both f16), row-major with K contiguous; C is
+// fp32 row-major.  A persistent kernel, one block per SM, walks 128 x 256 output
+// tiles.  Per tile the K dimension is cut in slices of 64: a producer thread
+// brings the A (128 x 64) and B (256 x 64) slices into a ring of shared-memory
+// stages with TMA tile loads (128-byte swizzle), one thread issues tcgen05.mma
+// (M = 128, N = 256, K = 16, four per slice) accumulating in tensor memory, and
+// four epilogue warps read the accumulator back with tcgen05.ld, scale it and
+// store it.  Two accumulators (2 x 256 TMEM columns) let the epilogue of one
+// tile overlap the MMAs of the next.
+//
+// Every wait on an mbarrier is bounded.  A wait that runs out records a code in
+// *status, raises a block-wide abort flag, and every role leaves its loop; the
+// block then lets its own copies land, frees its tensor memory and returns.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace dvp {
+namespace gemm {
+
+constexpr int kBM = 128, kBN = 256, kBK = 64;
+constexpr int kStages = 4;
+constexpr int kUmmaK = 16;
+constexpr int kThreads = 192;  // warp 0: TMA, warp 1: MMA, warps 2..5: epilogue
+constexpr uint32_t kBytesA = kBM * kBK * 2, kBytesB = kBN * kBK * 2;
+constexpr uint32_t kStageBytes = kBytesA + kBytesB;
+constexpr uint32_t kTmemCols = 512;
+constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kStages * kStageBytes + 256;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+enum { kErrNone = 0, kErrProducerWait = 11, kErrMmaWaitFull = 12, kErrMmaWaitTmem = 13,
+       kErrEpilogueWait = 14 };
+
+struct Params {
+  float *C;
+  long long ldc;
+  int M, N, K;
+  float alpha;
+  const float *alpha_dev;  // optional device scalar multiplied into alpha
+  int accumulate;          // C += instead of C =
+  int *status;             // device word, set non-zero when a wait gives up
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the limit ran out or another role raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (it > 32) __nanosleep(40);
+    if ((it & 255u) == 255u && *abort_flag) return false;
+  }
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x,
+                                            int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, "
+      "%4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of
+// 128 bytes, groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3ffffu) >> 4);  // start address
+  d |= (uint64_t)1 << 16;                   // leading byte offset (unused with swizzle): 16 B
+  d |= (uint64_t)(1024 >> 4) << 32;         // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                   // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                   // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor for kind::f16: fp32 accumulate, A and B of format
+// `fmt` (0 = f16, 1 = bf16), both K-major, M = 128, N = 256.
+__device__ __forceinline__ uint32_t instr_desc(uint32_t fmt) {
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kBN >> 3) << 17) |
+         ((uint32_t)(kBM >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                     uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_wait_ld() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+
+struct Shared {
+  uint64_t full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const Params p, const uint32_t fmt) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms are 1024-byte aligned
+  uint8_t *aligned = smem_raw + (base - smem_u32(smem_raw));
+  Shared *sh = reinterpret_cast<Shared *>(aligned + (size_t)kStages * kStageBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  const int tiles_m = (p.M + kBM - 1) / kBM, tiles_n = (p.N + kBN - 1) / kBN;
+  const int n_tiles = tiles_m * tiles_n;
+  const int k_slices = (p.K + kBK - 1) / kBK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&sh->full[s]), 1);
+      mbar_init(smem_u32(&sh->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&sh->tmem_full[b]), 1);
+      mbar_init(smem_u32(&sh->tmem_empty[b]), 4);
+    }
+    sh->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // one warp allocates the tensor memory of the block
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(&sh->tmem_base)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = sh->tmem_base;
+  volatile int *abort_flag = &sh->abort_flag;
+
+  if (warp == 0) {
+    // ---------------- producer: TMA loads into the stage ring
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x) {
+        const int tm = tile % tiles_m, tn = tile / tiles_m;
+        for (int ks = 0; ks < k_slices; ++ks, ++it) {
+          const uint32_t s = it % kStages, round = it / kStages;
+          if (round > 0 && !mbar_wait(smem_u32(&sh->empty[s]), (round - 1) & 1, abort_flag)) {
+            if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, kErrProducerWait); }
+            break;
+          }
+          const uint32_t bar = smem_u32(&sh->full[s]);
+          mbar_expect_tx(bar, kStageBytes);
+          const uint32_t dst = base + s * kStageBytes;
+          tma_load_2d(dst, &map_a, bar, ks * kBK, tm * kBM);
+          tma_load_2d(dst + kBytesA, &map_b, bar, ks * kBK, tn * kBN);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(fmt);
+      uint32_t it = 0, local_tile = 0;
+      for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x, ++local_tile) {
+        const uint32_t buf = local_tile & 1, use = local_tile >> 1;
+        if (use > 0 && !mbar_wait(smem_u32(&sh->tmem_empty[buf]), (use - 1) & 1, abort_flag)) {
+          if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, kErrMmaWaitTmem); }
+          break;
+        }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + buf * kBN;
+        bool ok = true;
+        for (int ks = 0; ks < k_slices; ++ks, ++it) {
+          const uint32_t s = it % kStages, round = it / kStages;
+          if (!mbar_wait(smem_u32(&sh->full[s]), round & 1, abort_flag)) {
+            if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, kErrMmaWaitFull); }
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t a_addr = base + s * kStageBytes, b_addr = a_addr + kBytesA;
+          const uint64_t adesc = smem_desc_sw128(a_addr), bdesc = smem_desc_sw128(b_addr);
+#pragma unroll
+          for (int k = 0; k < kBK / kUmmaK; ++k) {
+            // 16 elements of K are 32 bytes inside the 128-byte swizzled row
+            const uint64_t step = (uint64_t)((k * kUmmaK * 2) >> 4);
+            umma(tmem_d, adesc + step, bdesc + step, idesc, (ks > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(smem_u32(&sh->empty[s]));  // the stage is free once these MMAs have read it
+        }
+        if (!ok) break;
+        umma_commit(smem_u32(&sh->tmem_full[buf]));  // accumulator complete
+      }
+    }
+  } else {
+    // ---------------- epilogue: TMEM -> registers -> global
+    const int quarter = warp & 3;  // TMEM lanes this warp may read
+    const float alpha = p.alpha * (p.alpha_dev ? *p.alpha_dev : 1.f);
+    uint32_t local_tile = 0;
+    for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x, ++local_tile) {
+      const int tm = tile % tiles_m, tn = tile / tiles_m;
+      const uint32_t buf = local_tile & 1, use = local_tile >> 1;
+      if (!mbar_wait(smem_u32(&sh->tmem_full[buf]), use & 1, abort_flag)) {
+        if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, kErrEpilogueWait); }
+        break;
+      }
+      tc_fence_after();
+      const int row = tm * kBM + quarter * 32 + lane;
+      float *crow = p.C + (long long)row * p.ldc;
+#pragma unroll 1
+      for (int c0 = 0; c0 < kBN; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kBN + c0, r);
+        tmem_wait_ld();
+        const int col = tn * kBN + c0;
+        if (row < p.M && col < p.N) {
+          if (col + 32 <= p.N) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              uint32_t w[8];
+              if (p.accumulate) {
+                const float4 o0 = *reinterpret_cast<const float4 *>(crow + col + j);
+                const float4 o1 = *reinterpret_cast<const float4 *>(crow + col + j + 4);
+                const float old[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                  w[e] = __float_as_uint(fmaf(alpha, __uint_as_float(r[j + e]), old[e]));
+              } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) w[e] = __float_as_uint(alpha * __uint_as_float(r[j + e]));
+              }
+              asm volatile("st.global.v8.u32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(crow + col + j),
+                           "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]),
+                           "r"(w[7])
+                           : "memory");
+            }
+          } else {
+            for (int j = 0; j < 32 && col + j < p.N; ++j) {
+              const float v = alpha * __uint_as_float(r[j]);
+              crow[col + j] = p.accumulate ? crow[col + j] + v : v;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[buf]));
+    }
+  }
+
+  // ---------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0) {
+    // give this block's copies in flight time to land before the memory is released
+    for (int i = 0; i < 2000; ++i) __nanosleep(500);
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols)
+                 : "memory");
+  }
+}
+
+// ---- host side ------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// Tensor map of a row-major [rows, k] 16-bit matrix (row stride ld elements)
+// for boxes of box_rows x 64 with the 128-byte swizzle; reads past the extents
+// return zeros.
+inline bool make_map(CUtensorMap *map, const void *base, long long rows, long long k, long long ld,
+                     int box_rows, bool is_bf16) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)k, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2,
+            const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// C[M,N] (+)= alpha * A[M,K] * B[N,K]^T.  lda, ldb multiples of 8; ldc of 8; bases 16-byte
+// (A, B) and 32-byte (C) aligned.  Returns a CUDA error code; cudaErrorInvalidValue for
+// layouts it cannot take.
+inline cudaError_t launch_gemm_tn(const void *A, long long lda, const void *B, long long ldb, float *C,
+                                  long long ldc, int M, int N, int K, bool is_bf16, float alpha,
+                                  const float *alpha_dev, bool accumulate, int *status, int sm_count,
+                                  cudaStream_t stream) {
+  if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
+  if (lda % 8 || ldb % 8 || ldc % 8 || (uintptr_t)A % 16 || (uintptr_t)B % 16 || (uintptr_t)C % 32)
+    return cudaErrorInvalidValue;
+  CUtensorMap map_a, map_b;
+  if (!make_map(&map_a, A, M, K, lda, kBM, is_bf16) || !make_map(&map_b, B, N, K, ldb, kBN, is_bf16))
+    return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(gemm_tn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)kSmemBytes);
+  if (e != cudaSuccess) return e;
+  Params p{C, ldc, M, N, K, alpha, alpha_dev, accumulate ? 1 : 0, status};
+  const int tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
+  const int grid = tiles < sm_count ? tiles : sm_count;
+  gemm_tn_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, p, is_bf16 ? 1u : 0u);
+  return cudaGetLastError();
+}
+
+}  // namespace gemm
+}  // namespace dvp

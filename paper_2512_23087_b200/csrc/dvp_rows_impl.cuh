@@ -422,7 +422,7 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
       row_stats<TIn, kStage>(trow, V, a, p.log_rho, bound, scratch, hot_smem, hot, mask_t);
 
   if (p.grad) {
-    const float g = p.upstream[t];
+    const float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
     row_grad<TIn, TGrad, kStage>(trow, reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad, V, a, st,
                                  g, bound, hot);
   }
@@ -513,7 +513,7 @@ __global__ void dvp_row_kernel_scalar(const RowParams p) {
 
   if (p.grad) {
     TGrad *grow = reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad;
-    const float g = p.upstream[t];
+    const float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
     const float s_safe = st.s_x + st.e_a;
     const bool live = st.member;
     const float coef = live ? -g / s_safe : 0.f;

@@ -1,0 +1,180 @@
+"""Parity of the tensor-core contraction and of the fused LM-head entry point
+with the fp64 oracle, through the C ABI.
+
+Membership in the fused variant is decided on bf16 x bf16 products accumulated
+in fp32 by the tensor cores (H/16 accumulation steps, each good to one unit in
+the last place of the running sum), so it cannot be bit-exact against fp64
+logits: rows that hold a logit within (H/16 + 2) 2^-24 max|z| + 1e-6 of the
+threshold are counted and compared on log-probabilities only (their safe-set
+size may differ by at most the number of such logits); every other row is
+compared exactly like the row kernels.
+Gradients: per token row of d_hidden and per vocabulary row of d_w,
+||X - X_oracle||_2 <= 1e-3 ||X_oracle||_2 + 1e-6 * (largest row norm), the second
+term covering rows that are zero up to the float16 grid of the gradient panel.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2512_23087_b200 import binding, inputs
+
+import parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _bits(x):
+    return x.detach().cpu().view(torch.int16).numpy().view(np.uint16)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("m,n,k", [(128, 256, 64), (128, 256, 512), (300, 520, 200), (1, 8, 8),
+                                   (1000, 776, 1032), (257, 4096, 4104), (2048, 512, 8192)])
+def test_gemm_tn_matches_float64_matmul(dtype, m, n, k):
+    g = torch.Generator(device=DEV).manual_seed(m * 7 + n * 3 + k)
+    a = torch.randn(m, k, generator=g, device=DEV).to(dtype)
+    b = torch.randn(n, k, generator=g, device=DEV).to(dtype)
+    ref = (a.double() @ b.double().t())
+    out, status = binding.dvp_gemm_tn(a, b, alpha=0.5)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    # fp32 accumulation in tensor memory: up to one unit in the last place per 16-wide step
+    tol = (2.0 ** -24 * (k / 16) + 1e-6) * ref.abs().max().item()
+    err = (out.double() - 0.5 * ref).abs().max().item()
+    assert err <= tol, (err, tol)
+    # accumulate on top, strided operands, misaligned-free views
+    out2, status = binding.dvp_gemm_tn(a, b, alpha=0.25, out=out.clone(), accumulate=True)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert (out2.double() - 0.75 * ref).abs().max().item() <= 2 * tol
+
+
+def test_gemm_tn_padded_strides_and_argument_errors():
+    g = torch.Generator(device=DEV).manual_seed(5)
+    a = torch.randn(200, 328, generator=g, device=DEV).to(torch.bfloat16)[:, :320]
+    b = torch.randn(130, 336, generator=g, device=DEV).to(torch.bfloat16)[:, :320]
+    out = torch.full((200, 136), 7.0, device=DEV)[:, :130]
+    binding.dvp_gemm_tn(a, b, out=out)
+    torch.cuda.synchronize()
+    ref = a.double() @ b.double().t()
+    assert (out.double() - ref).abs().max().item() < 1e-3
+    with pytest.raises(binding.DvpError) as e:
+        binding.dvp_gemm_tn(a[:, :317], b[:, :317].contiguous())      # lda = 328 ok, ldb = 317 not
+    assert e.value.status == binding.DVP_ERR_UNSUPPORTED
+
+
+def _check_fused(batch, rho, res, want, V):
+    rep = {}
+    z = want.logits
+    H = batch.hidden.shape[1]
+    for label, got, side, logits in (("train", res.train, want.rows.train, z),
+                                     ("infer", res.infer, want.rows.infer, None)):
+        if got is None:
+            continue
+        if logits is None:
+            logits = batch.infer.detach().cpu().double().numpy()
+        tau = side.tau[:, None]
+        width = (H / 16 + 2) * 2.0 ** -24 * np.abs(logits).max(axis=1, keepdims=True) + 1e-6
+        band = np.abs(logits - tau) <= width
+        band_rows = band.any(axis=1) if label == "train" else np.zeros(len(tau), dtype=bool)
+        ok = ~band_rows
+        rep[f"{label}_band_rows"] = int(band_rows.sum())
+        cnt = got.count.cpu().numpy().astype(np.int64)
+        assert np.array_equal(cnt[ok], side.count[ok]), f"{label}.count"
+        assert (np.abs(cnt - side.count) <= band.sum(axis=1))[band_rows].all()
+        np.testing.assert_allclose(got.max.cpu().numpy(), side.max, atol=1e-4, rtol=0)
+        np.testing.assert_allclose(got.lse.cpu().numpy(), side.lse, atol=1e-4, rtol=0)
+        np.testing.assert_allclose(got.lse_safe.cpu().numpy(), side.lse_safe, atol=1e-4, rtol=0)
+        np.testing.assert_allclose(got.logp.cpu().numpy(), side.logp, atol=1e-4, rtol=0)
+        lp = got.logp_mp.cpu().numpy().astype(np.float64)
+        assert np.array_equal(np.isneginf(lp)[ok], np.isneginf(side.logp_mp)[ok])
+        fin = np.isfinite(side.logp_mp) & np.isfinite(lp)
+        assert np.abs(lp[fin] - side.logp_mp[fin]).max() <= 1e-4
+        rep[f"{label}_ok"] = ok
+    ok = rep["train_ok"]
+    flags = res.flags.cpu().numpy()
+    assert np.array_equal((flags & 1)[ok], want.rows.train.member[ok])
+    if res.infer is not None:
+        assert np.array_equal((flags >> 1) & 1, want.rows.infer.member)
+        lr = res.log_ratio.cpu().numpy().astype(np.float64)
+        wl = want.rows.log_ratio
+        fin = np.isfinite(wl) & ok
+        assert np.abs(lr[fin] - wl[fin]).max() <= 2e-4
+        assert np.array_equal(np.isinf(lr)[ok], np.isinf(wl)[ok])
+
+    def rows_close(got, ref, name, rows=None):
+        got = got.cpu().double().numpy()
+        if rows is not None:
+            got, ref = got[rows], ref[rows]
+        num = np.sqrt(((got - ref) ** 2).sum(axis=1))
+        den = np.sqrt((ref ** 2).sum(axis=1))
+        bound = 1e-3 * den + 1e-6 * den.max()
+        assert (num <= bound).all(), f"{name}: worst {np.max(num / np.maximum(den, 1e-300)):.3e}"
+        rep[name] = float(np.max(num / np.maximum(den, 1e-6 * den.max())))
+
+    rows_close(res.d_hidden, want.d_hidden, "d_hidden", ok)
+    if ok.all():
+        rows_close(res.d_w, want.d_w, "d_w")
+    return rep
+
+
+def _run_fused(T, H, V, rho, seed, **kw):
+    w = inputs.WORKLOADS["c4_fused_lmhead"]
+    batch = inputs.make_fused(w, seed=seed, device=DEV, T=T, H=H, V=V)
+    res = binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, rho,
+                                                    batch.upstream, infer_logits=batch.infer, **kw)
+    torch.cuda.synchronize()
+    assert res.workspace[:4].view(torch.int32).item() == 0, "a tensor-core kernel gave up waiting"
+    want = oracle.dvp_fused_lmhead(_bits(batch.hidden), _bits(batch.w_vocab), _bits(batch.infer),
+                                   batch.ids.cpu().numpy(), rho, batch.upstream.cpu().numpy().astype(np.float64))
+    return batch, res, want
+
+
+@pytest.mark.parametrize("T,H,V,rho", [(200, 256, 3000, 1e-3), (64, 128, 1000, 1e-2), (130, 512, 5008, 1e-4),
+                                       (128, 4096, 4096, 1e-3)])
+def test_fused_lmhead_small(T, H, V, rho):
+    batch, res, want = _run_fused(T, H, V, rho, seed=T)
+    _check_fused(batch, rho, res, want, V)
+
+
+def test_fused_lmhead_several_panels_and_dw_accumulation():
+    T, H, V, rho = 300, 256, 2048, 1e-3
+    w = inputs.WORKLOADS["c4_fused_lmhead"]
+    batch = inputs.make_fused(w, seed=9, device=DEV, T=T, H=H, V=V)
+    d_w = torch.full((V, H), 0.5, device=DEV)
+    res = binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, rho,
+                                                    batch.upstream, infer_logits=batch.infer,
+                                                    panel_rows=128, d_w=d_w, accumulate_dw=True)
+    torch.cuda.synchronize()
+    assert res.workspace[:4].view(torch.int32).item() == 0
+    want = oracle.dvp_fused_lmhead(_bits(batch.hidden), _bits(batch.w_vocab), _bits(batch.infer),
+                                   batch.ids.cpu().numpy(), rho, batch.upstream.cpu().numpy().astype(np.float64))
+    want.d_w += 0.5
+    rep = _check_fused(batch, rho, res, want, V)
+    one = binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, rho,
+                                                    batch.upstream, infer_logits=batch.infer)
+    torch.cuda.synchronize()
+    assert (one.d_hidden - res.d_hidden).abs().max().item() <= 1e-5 * res.d_hidden.abs().max().item()
+    assert torch.equal(one.train.count, res.train.count)
+
+
+def test_fused_lmhead_full_vocabulary_rows():
+    """V = 151,936 with the LM-head statistics of the benchmark configuration."""
+    batch, res, want = _run_fused(256, 1024, 151936, 1e-3, seed=3)
+    rep = _check_fused(batch, 1e-3, res, want, 151936)
+    assert want.rows.train.count.mean() > 1000        # dense safe sets, as in the full configuration
+
+
+def test_fused_argument_errors():
+    w = inputs.WORKLOADS["c4_fused_lmhead"]
+    batch = inputs.make_fused(w, seed=1, device=DEV, T=16, H=64, V=256)
+    with pytest.raises(binding.DvpError) as e:
+        binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, 1e-3,
+                                                  batch.upstream, panel_rows=100)
+    assert e.value.status == binding.DVP_ERR_INVALID_ARG
+    with pytest.raises(binding.DvpError) as e:
+        binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, 1e-3,
+                                                  batch.upstream, workspace=torch.empty(512, dtype=torch.uint8, device=DEV))
+    assert e.value.status == binding.DVP_ERR_WORKSPACE
