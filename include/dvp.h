@@ -229,6 +229,48 @@ typedef struct {
 int dvp_fused_lmhead_forward_backward(const dvp_fused_args *args);
 
 /*
+ * dvp_fused_lmhead_forward_backward_static -- the fused entry point for callers
+ * that cannot obtain device memory of their own.  (The paper has no counterpart;
+ * this is a packaging variant of the entry point above.)
+ *
+ * Who needs it: code that runs inside a host application which hands out all
+ * device memory up front and forbids further allocation, code on a latency
+ * critical path where an allocator call (which may synchronise the whole
+ * device) is not acceptable, and code that is simply not allowed to own
+ * buffers between calls.  Such a caller has the inputs and outputs it was given
+ * but no place to put a workspace, and the fused computation cannot run
+ * without one.
+ *
+ * What it does: exactly dvp_fused_lmhead_forward_backward, except that
+ * `workspace` and `workspace_bytes` are ignored and the workspace is a fixed
+ * array of DVP_STATIC_WORKSPACE_BYTES (32 MiB) that is part of the library
+ * image.  Every GPU on which the library's code is loaded holds those 32 MiB
+ * until the process exits, whether or not this function is ever called.
+ * `panel_rows` = 0 selects 128 here.  The call itself allocates and frees
+ * nothing, on the device or through any library.
+ *
+ * Limit: the workspace the arguments need (dvp_workspace_bytes with the same
+ * panel_rows; roughly (2 H + 8 panel_rows) V + 2 H T bytes) must fit in
+ * DVP_STATIC_WORKSPACE_BYTES, e.g. H = 1024, V = 8192, any T up to a few
+ * thousand.  Larger problems return DVP_ERR_WORKSPACE and launch nothing.
+ * Other errors are those of dvp_fused_lmhead_forward_backward;
+ * DVP_ERR_UNSUPPORTED also for a device ordinal of 64 or more.
+ *
+ * First call on each device: it looks up the array's device address (once per
+ * device, with that device current).  Make that first call outside any stream
+ * capture.
+ *
+ * Sharing: all calls on one GPU use the same array, and the array keeps
+ * whatever the previous call left in it (the library resets the one word that
+ * has to start at zero).  Two calls whose kernels can overlap on the GPU (for
+ * instance on different streams) race on it and corrupt each other; issue such
+ * calls on one stream, or order them yourself.  After the stream has finished,
+ * nothing in the array is needed any more.
+ */
+#define DVP_STATIC_WORKSPACE_BYTES (32u * 1024u * 1024u)
+int dvp_fused_lmhead_forward_backward_static(const dvp_fused_args *args);
+
+/*
  * dvp_gemm_tn -- the tensor-core contraction the fused entry point is built on,
  * exposed for reuse and testing: C[m, n] (+)= alpha * A[m, k] * B[n, k]^T with A
  * and B both bf16 or both f16 (dtype), row-major with k contiguous, C float32

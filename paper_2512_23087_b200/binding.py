@@ -21,8 +21,10 @@ DVP_F32, DVP_BF16, DVP_F16 = 0, 1, 2
 DVP_ID_I64, DVP_ID_I32 = 0, 1
 DVP_FLAG_IN_TRAIN, DVP_FLAG_IN_INFER, DVP_FLAG_NO_ID, DVP_FLAG_BAD_ID = 1, 2, 64, 128
 DVP_ENTRY_FORWARD, DVP_ENTRY_BACKWARD, DVP_ENTRY_FUSED_LMHEAD = 0, 1, 2
+DVP_STATIC_WORKSPACE_BYTES = 32 * 1024 * 1024
 
-EXPORTS = ("dvp_forward", "dvp_backward", "dvp_fused_lmhead_forward_backward", "dvp_gemm_tn",
+EXPORTS = ("dvp_forward", "dvp_backward", "dvp_fused_lmhead_forward_backward",
+           "dvp_fused_lmhead_forward_backward_static", "dvp_gemm_tn",
            "dvp_workspace_bytes", "dvp_status_string", "dvp_version")
 
 _DTYPES = {torch.float32: DVP_F32, torch.bfloat16: DVP_BF16, torch.float16: DVP_F16}
@@ -141,6 +143,8 @@ def load_library() -> ctypes.CDLL:
         lib.dvp_backward.restype = ctypes.c_int
         lib.dvp_fused_lmhead_forward_backward.argtypes = [ctypes.POINTER(FusedArgs)]
         lib.dvp_fused_lmhead_forward_backward.restype = ctypes.c_int
+        lib.dvp_fused_lmhead_forward_backward_static.argtypes = [ctypes.POINTER(FusedArgs)]
+        lib.dvp_fused_lmhead_forward_backward_static.restype = ctypes.c_int
         lib.dvp_gemm_tn.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64,
                                     ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int64, ctypes.c_int32, ctypes.c_float, ctypes.c_int32,
@@ -366,4 +370,58 @@ def dvp_fused_lmhead_forward_backward(hidden: torch.Tensor, w_vocab: torch.Tenso
     st = lib.dvp_fused_lmhead_forward_backward(ctypes.byref(a))
     if st != DVP_OK:
         raise DvpError(st, "dvp_fused_lmhead_forward_backward")
+    return res
+
+
+def dvp_fused_lmhead_forward_backward_static(hidden: torch.Tensor, w_vocab: torch.Tensor,
+                                             ids: torch.Tensor, rho: float, upstream: torch.Tensor, *,
+                                             infer_logits: torch.Tensor | None = None,
+                                             d_w: torch.Tensor | None = None,
+                                             accumulate_dw: bool = False, panel_rows: int = 0,
+                                             stream=None):
+    """The fused LM-head computation for callers that have no device memory of
+    their own to offer as a workspace: the library uses a fixed 32 MiB array that
+    is part of its image instead, and the call allocates nothing (this wrapper
+    only creates the output tensors a caller would normally already own).
+
+    Problems whose workspace would not fit raise ``DvpError`` with
+    ``DVP_ERR_WORKSPACE``.  All calls on a GPU share that one array, so calls
+    that could overlap on the GPU (different streams) must be ordered by the
+    caller.  Make the first call on each device outside any stream capture."""
+    lib = load_library()
+    _check_matrix("hidden", hidden)
+    _check_matrix("w_vocab", w_vocab)
+    T, H = hidden.shape
+    V = w_vocab.shape[0]
+    dev = hidden.device
+    if hidden.dtype != torch.bfloat16 or w_vocab.dtype != torch.bfloat16:
+        raise TypeError("hidden and w_vocab must be bfloat16")
+    a = FusedArgs()
+    a.struct_size = ctypes.sizeof(FusedArgs)
+    a.id_dtype = _id_dtype(ids)
+    a.T, a.H, a.V, a.rho = T, H, V, float(rho)
+    a.ld_hidden, a.ld_w = hidden.stride(0), w_vocab.stride(0)
+    a.hidden, a.w_vocab, a.ids, a.upstream = _ptr(hidden), _ptr(w_vocab), _ptr(ids), _ptr(upstream)
+    res = SimpleNamespace(infer=None, log_ratio=None)
+    res.train, a.train = _side(dev, T, V, False)
+    res.flags = torch.empty(T, dtype=torch.uint8, device=dev)
+    a.flags = _ptr(res.flags)
+    if infer_logits is not None:
+        _check_matrix("infer_logits", infer_logits)
+        if infer_logits.dtype != torch.bfloat16:
+            raise TypeError("infer_logits must be bfloat16")
+        a.infer_logits, a.ld_infer = _ptr(infer_logits), infer_logits.stride(0)
+        res.infer, a.infer = _side(dev, T, V, False)
+        res.log_ratio = torch.empty(T, dtype=torch.float32, device=dev)
+        a.log_ratio = _ptr(res.log_ratio)
+    res.d_hidden = torch.empty(T, H, dtype=torch.float32, device=dev)
+    res.d_w = d_w if d_w is not None else torch.empty(V, H, dtype=torch.float32, device=dev)
+    a.d_hidden, a.ld_dh = _ptr(res.d_hidden), res.d_hidden.stride(0)
+    a.d_w, a.ld_dw = _ptr(res.d_w), res.d_w.stride(0)
+    a.accumulate_dw = int(accumulate_dw)
+    a.panel_rows = int(panel_rows)
+    a.stream = _stream(stream)
+    st = lib.dvp_fused_lmhead_forward_backward_static(ctypes.byref(a))
+    if st != DVP_OK:
+        raise DvpError(st, "dvp_fused_lmhead_forward_backward_static")
     return res

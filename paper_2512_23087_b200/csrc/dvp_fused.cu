@@ -15,6 +15,7 @@
 // converted to float16 copies once per call (exact for bfloat16 values in
 // float16's normal range).
 #include <cmath>
+#include <mutex>
 
 #include "dvp_common.cuh"
 #include "dvp_gemm.cuh"
@@ -274,6 +275,50 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
                                                                         a->log_ratio);
   }
   return cudaGetLastError() == cudaSuccess ? DVP_OK : DVP_ERR_CUDA;
+}
+
+
+// ---- a variant that allocates nothing ------------------------------------------
+// The workspace of the fused entry point, taken from a fixed array that is part
+// of the loaded library instead of from the caller.  In host code the array's
+// name is only a handle; the device address comes from cudaGetSymbolAddress, once
+// per device, with that device current.
+
+}  // extern "C"
+
+namespace {
+constexpr size_t kStaticWorkspaceBytes = (size_t)DVP_STATIC_WORKSPACE_BYTES;
+static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes];
+constexpr int kMaxDevices = 64;
+void *g_static_workspace_ptr[kMaxDevices] = {};
+std::mutex g_static_workspace_mutex;
+}  // namespace
+
+extern "C" {
+
+int dvp_fused_lmhead_forward_backward_static(const dvp_fused_args *a) {
+  if (!a || a->struct_size != sizeof(dvp_fused_args)) return DVP_ERR_INVALID_ARG;
+  dvp_fused_args b = *a;
+  if (b.panel_rows == 0) b.panel_rows = 128;  // the smallest panel leaves the most room
+  dvp::FusedLayout L;
+  if (!dvp::fused_layout(&b, &L)) return DVP_ERR_INVALID_ARG;
+  if (L.total > kStaticWorkspaceBytes) return DVP_ERR_WORKSPACE;  // beyond the built-in maximum
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return DVP_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return DVP_ERR_UNSUPPORTED;
+  void *ptr = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_workspace_mutex);
+    if (!g_static_workspace_ptr[dev]) {
+      void *sym = nullptr;
+      if (cudaGetSymbolAddress(&sym, g_static_workspace) != cudaSuccess || !sym) return DVP_ERR_CUDA;
+      g_static_workspace_ptr[dev] = sym;
+    }
+    ptr = g_static_workspace_ptr[dev];
+  }
+  b.workspace = ptr;
+  b.workspace_bytes = kStaticWorkspaceBytes;
+  return dvp_fused_lmhead_forward_backward(&b);
 }
 
 }  // extern "C"
