@@ -161,6 +161,9 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int tiles_m = (p.M + kBM - 1) / kBM, tiles_n = (p.N + kBN - 1) / kBN;
   const int n_tiles = tiles_m * tiles_n;
   const int k_slices = (p.K + kBK - 1) / kBK;
+  // Blocks that run together take consecutive tiles: walk the shorter tile dimension
+  // fastest so that they share the operand panel of the longer one through L2.
+  const bool m_fastest = tiles_m <= tiles_n;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -192,7 +195,8 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (lane == 0) {
       uint32_t it = 0;
       for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x) {
-        const int tm = tile % tiles_m, tn = tile / tiles_m;
+        const int tm = m_fastest ? tile % tiles_m : tile / tiles_n;
+        const int tn = m_fastest ? tile / tiles_m : tile % tiles_n;
         for (int ks = 0; ks < k_slices; ++ks, ++it) {
           const uint32_t s = it % kStages, round = it / kStages;
           if (round > 0 && !mbar_wait(smem_u32(&sh->empty[s]), (round - 1) & 1, abort_flag)) {
@@ -249,7 +253,8 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const float alpha = p.alpha * (p.alpha_dev ? *p.alpha_dev : 1.f);
     uint32_t local_tile = 0;
     for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x, ++local_tile) {
-      const int tm = tile % tiles_m, tn = tile / tiles_m;
+      const int tm = m_fastest ? tile % tiles_m : tile / tiles_n;
+      const int tn = m_fastest ? tile / tiles_m : tile % tiles_n;
       const uint32_t buf = local_tile & 1, use = local_tile >> 1;
       if (!mbar_wait(smem_u32(&sh->tmem_full[buf]), use & 1, abort_flag)) {
         if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, kErrEpilogueWait); }
