@@ -22,21 +22,60 @@
 
 namespace dvp {
 
-// out[c, r] = convert(in[r, c]) for a row-major [R, C] input.
+// out[c, r] = convert(in[r, c]) for a row-major [R, C] input of a 16-bit type.
+// 64 x 64 tiles through shared memory; 16-byte accesses on both sides when the
+// strides and bases allow it (ld_in, ld_out multiples of 8, 16-byte aligned bases).
 template <typename TIn, typename TOut>
-__global__ void transpose_convert_kernel(const TIn *in, long long ld_in, TOut *out, long long ld_out,
-                                         int R, int C) {
-  __shared__ float tile[32][33];
-  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
-  for (int j = threadIdx.y; j < 32; j += blockDim.y) {
-    const int r = r0 + j, c = c0 + threadIdx.x;
-    tile[j][threadIdx.x] = (r < R && c < C) ? Storage<TIn>::widen(in[(long long)r * ld_in + c]) : 0.f;
+__global__ void __launch_bounds__(256)
+transpose_convert_kernel(const TIn *in, long long ld_in, TOut *out, long long ld_out, int R, int C,
+                         int vec_ok) {
+  __shared__ TOut tile[64][66];
+  const int c0 = blockIdx.x * 64, r0 = blockIdx.y * 64;
+  const int tid = threadIdx.x;
+  // load: 64 rows x 8 vectors of 8 elements, two vectors per thread
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int v = tid + i * 256, r = r0 + (v >> 3), c = c0 + (v & 7) * 8;
+    TOut e[8];
+    if (vec_ok && r < R && c + 8 <= C) {
+      const uint4 raw = *reinterpret_cast<const uint4 *>(in + (long long)r * ld_in + c);
+      const TIn *x = reinterpret_cast<const TIn *>(&raw);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) e[j] = Storage<TOut>::narrow(Storage<TIn>::widen(x[j]));
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        e[j] = (r < R && c + j < C)
+                   ? Storage<TOut>::narrow(Storage<TIn>::widen(in[(long long)r * ld_in + c + j]))
+                   : Storage<TOut>::narrow(0.f);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) tile[v >> 3][(v & 7) * 8 + j] = e[j];
   }
   __syncthreads();
-  for (int j = threadIdx.y; j < 32; j += blockDim.y) {
-    const int c = c0 + j, r = r0 + threadIdx.x;
-    if (c < C && r < R) out[(long long)c * ld_out + r] = Storage<TOut>::narrow(tile[threadIdx.x][j]);
+  // store: 64 output rows (input columns) x 8 vectors of 8 input rows
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int v = tid + i * 256, c = c0 + (v >> 3), r = r0 + (v & 7) * 8;
+    if (c >= C) continue;
+    __align__(16) TOut e[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) e[j] = tile[(v & 7) * 8 + j][v >> 3];
+    TOut *dst = out + (long long)c * ld_out + r;
+    if (vec_ok && r + 8 <= R) {
+      *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(e);
+    } else {
+      for (int j = 0; j < 8 && r + j < R; ++j) dst[j] = e[j];
+    }
   }
+}
+
+template <typename TIn, typename TOut>
+static void launch_transpose(const TIn *in, long long ld_in, TOut *out, long long ld_out, int R, int C,
+                             cudaStream_t s) {
+  const int vec_ok = ld_in % 8 == 0 && ld_out % 8 == 0 && (uintptr_t)in % 16 == 0 && (uintptr_t)out % 16 == 0;
+  transpose_convert_kernel<TIn, TOut>
+      <<<dim3((C + 63) / 64, (R + 63) / 64), 256, 0, s>>>(in, ld_in, out, ld_out, R, C, vec_ok);
 }
 
 struct FusedScalars {
@@ -213,11 +252,8 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
   const long long mask_words = (a->V + 31) / 32;
 
   grad_scale_kernel<<<1, 1024, 0, s>>>(a->upstream, a->T, sc);
-  const dim3 tb(32, 8);
-  transpose_convert_kernel<__nv_bfloat16, __half>
-      <<<dim3((H + 31) / 32, (V + 31) / 32), tb, 0, s>>>(w, a->ld_w, wt16, L.Vp, V, H);
-  transpose_convert_kernel<__nv_bfloat16, __half>
-      <<<dim3((H + 31) / 32, (T + 31) / 32), tb, 0, s>>>(hidden, a->ld_hidden, ht16, L.Tp, T, H);
+  launch_transpose<__nv_bfloat16, __half>(w, a->ld_w, wt16, L.Vp, V, H, s);
+  launch_transpose<__nv_bfloat16, __half>(hidden, a->ld_hidden, ht16, L.Tp, T, H, s);
   if (cudaGetLastError() != cudaSuccess) return DVP_ERR_CUDA;
 
   const double log_rho = a->rho > 0.0 ? std::log(a->rho) : -HUGE_VAL;
@@ -245,8 +281,7 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
     p.out_t.logp_mp = lpt + r0;
     p.flags = flt + r0;
     if (launch_row_kernels(p, DVP_F32, DVP_F16, 0, s) != cudaSuccess) return DVP_ERR_CUDA;
-    transpose_convert_kernel<__half, __half>
-        <<<dim3((V + 31) / 32, (rows + 31) / 32), tb, 0, s>>>(g16, L.Vp, gt16, L.panel, rows, V);
+    launch_transpose<__half, __half>(g16, L.Vp, gt16, L.panel, rows, V, s);
     // d_hidden[r0 : r0 + rows] = G x W / scale
     e = gemm::launch_gemm_tn(g16, L.Vp, wt16, L.Vp, a->d_hidden + r0 * a->ld_dh, a->ld_dh, rows, H, V,
                              false, 1.f, &sc->inv_scale, false, &sc->status, sms, s);
