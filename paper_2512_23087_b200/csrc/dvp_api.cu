@@ -10,7 +10,8 @@ bool dtype_ok(int d) { return d == DVP_F32 || d == DVP_BF16 || d == DVP_F16; }
 bool hint_ok(uint32_t hint) {
   const uint32_t threads = hint & 0xffff, stage = (hint >> 16) & 0xff;
   if (threads != 0 && (threads % 32 != 0 || threads > 512)) return false;
-  return (stage == 0 || stage == 1 || stage == 2) && (hint >> 24) == 0;
+  const uint32_t cluster = (hint >> 24) & 0xff;
+  return (stage == 0 || stage == 1 || stage == 2) && (cluster == 0 || cluster == 1 || cluster == 2 || cluster == 4);
 }
 
 bool side_empty(const dvp_side_out &o) {

@@ -257,21 +257,79 @@ __device__ __forceinline__ void absorb_stage(const Stage<TIn, kStage> &st, int s
   }
 }
 
-// Sweeps 1 and 2 over one row: statistics of one side.
+// ---- a row split over a thread-block cluster -----------------------------------
+// With kCluster > 1 the blocks of a cluster share one row: block `rank` owns a
+// contiguous part of it, partial results meet through distributed shared memory.
+// Fewer rows are then in flight (one per cluster instead of one per block), so
+// the granules that sweeps 2 and 3 revisit are still in L2.
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(const float *local, uint32_t rank) {
+  uint32_t laddr = (uint32_t)__cvta_generic_to_shared(local), raddr;
+  float v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(laddr), "r"(rank));
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(raddr) : "memory");
+  return v;
+}
+
+// slot: 4 floats of this block's shared memory, written once per kernel.
+template <int kCluster>
+__device__ __forceinline__ LogSum cluster_reduce_logsum(LogSum v, float *slot) {
+  if constexpr (kCluster == 1) return v;
+  if (threadIdx.x == 0) {
+    slot[0] = v.m;
+    slot[1] = v.c;
+    slot[2] = v.s;
+  }
+  cluster_sync_all();
+  LogSum r = {kNegInf, kNegInf, 0.f};
+#pragma unroll
+  for (uint32_t k = 0; k < (uint32_t)kCluster; ++k) {  // rank order: same result in every block
+    LogSum o;
+    o.m = ld_cluster_f32(slot + 0, k);
+    o.c = ld_cluster_f32(slot + 1, k);
+    o.s = ld_cluster_f32(slot + 2, k);
+    r = combine(r, o);
+  }
+  return r;
+}
+
+template <int kCluster>
+__device__ __forceinline__ SumCount cluster_reduce_sumcount(SumCount v, float *slot) {
+  if constexpr (kCluster == 1) return v;
+  if (threadIdx.x == 0) {
+    slot[0] = v.s;
+    slot[1] = __int_as_float(v.n);
+  }
+  cluster_sync_all();
+  SumCount r = {0.f, 0};
+#pragma unroll
+  for (uint32_t k = 0; k < (uint32_t)kCluster; ++k) {
+    r.s += ld_cluster_f32(slot + 0, k);
+    r.n += __float_as_int(ld_cluster_f32(slot + 1, k));
+  }
+  return r;
+}
+
+// Sweep 1 over (a part of) a row: block-wide log-sum-exp state; granule bounds
+// are left in shared memory.
 template <typename TIn, int kStage>
-__device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int a, double log_rho,
-                                               uint16_t *bound, float *scratch, uint32_t *hot_smem,
-                                               HotList &hot, uint32_t *mask_row) {
+__device__ __forceinline__ LogSum row_sweep1(const TIn *row, int V, uint16_t *bound, float *scratch) {
   constexpr int kElems = Granule<TIn>::kElems;
   const int n_full = V / kElems;
   const int n_gran = (V + kElems - 1) / kElems;
   const int per_step = kStage * (int)blockDim.x;
   const int n_steps = (n_gran + per_step - 1) / per_step;
-  const int tid = threadIdx.x;
-
-  // ---- sweep 1, two stages in flight
   LogSum acc = {kNegInf, kNegInf, 0.f};
-  {
+  if (n_steps > 0) {  // two stages in flight
     Stage<TIn, kStage> s0, s1;
     s0.load(row, V, n_full, 0);
     int step = 0;
@@ -283,21 +341,23 @@ __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int a, dou
     }
     if (step < n_steps) absorb_stage<TIn, kStage>(s0, step, acc, bound);
   }
-  const LogSum all = block_reduce_logsum(acc, scratch);
+  return block_reduce_logsum(acc, scratch);
+}
 
-  SideStats st;
-  st.m = all.m;
-  st.lse = lse_from_logsum(all);
-  st.tau = threshold_f32(all.m, log_rho);
-  const bool has_a = a >= 0 && a < V;
-  st.z_a = has_a ? Storage<TIn>::widen(row[a]) : 0.f;
-  st.member = has_a && st.z_a >= st.tau;
-  st.e_a = st.member ? ex2((st.z_a - st.m) * kLog2e) : 0.f;
-
-  // ---- sweep 2: only granules that can hold a safe token
+// Sweep 2 over (a part of) a row: masked sum without the sampled token and count,
+// block-wide.  `a` is relative to `row` (outside [0, V): not in this part).
+template <typename TIn, int kStage>
+__device__ __forceinline__ SumCount row_sweep2(const TIn *row, int V, int a, float tau, float m,
+                                               const uint16_t *bound, float *scratch,
+                                               uint32_t *hot_smem, HotList &hot) {
+  constexpr int kElems = Granule<TIn>::kElems;
+  const int n_full = V / kElems;
+  const int n_gran = (V + kElems - 1) / kElems;
+  const int per_step = kStage * (int)blockDim.x;
+  const int n_slots = ((n_gran + per_step - 1) / per_step) * kStage;  // granules per thread
+  const int tid = threadIdx.x;
   SumCount sc = {0.f, 0};
-  const int n_slots = n_steps * kStage;  // granules per thread
-  hot = build_hot_list(bound, n_slots, st.tau, hot_smem);
+  hot = build_hot_list(bound, n_slots, tau, hot_smem);
   if (hot.fits()) {
     const int wbase = tid & ~31, lane = tid & 31;
     for (int q = lane; q < hot.count; q += 64) {
@@ -309,27 +369,52 @@ __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int a, dou
       Granule<TIn> a0, a1;
       a0.load_any(row, V, n_full, g0);
       if (two) a1.load_any(row, V, n_full, g1);
-      granule_masked_sum<TIn>(a0, g0, a, st.tau, st.m, sc);
-      if (two) granule_masked_sum<TIn>(a1, g1, a, st.tau, st.m, sc);
+      granule_masked_sum<TIn>(a0, g0, a, tau, m, sc);
+      if (two) granule_masked_sum<TIn>(a1, g1, a, tau, m, sc);
     }
   } else {
     for (int i = 0; i < n_slots; ++i) {
-      if (bf16_bits_to_float(bound[i * blockDim.x + tid]) >= st.tau) {
+      if (bf16_bits_to_float(bound[i * blockDim.x + tid]) >= tau) {
         const int g = i * (int)blockDim.x + tid;
         Granule<TIn> gr;
         gr.load_any(row, V, n_full, g);
-        granule_masked_sum<TIn>(gr, g, a, st.tau, st.m, sc);
+        granule_masked_sum<TIn>(gr, g, a, tau, m, sc);
       }
     }
   }
-  const SumCount tot = block_reduce_sumcount(sc, scratch);
+  return block_reduce_sumcount(sc, scratch);
+}
+
+// Statistics of one side of one row.  `row` is the whole row (V elements); this
+// block sweeps the part [off, off + v_part) of it.
+template <typename TIn, int kStage, int kCluster>
+__device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int off, int v_part, int a,
+                                               double log_rho, uint16_t *bound, float *scratch,
+                                               float *cl_slots, uint32_t *hot_smem, HotList &hot,
+                                               uint32_t *mask_row) {
+  const LogSum part = row_sweep1<TIn, kStage>(row + off, v_part, bound, scratch);
+  const LogSum all = cluster_reduce_logsum<kCluster>(part, cl_slots);
+
+  SideStats st;
+  st.m = all.m;
+  st.lse = lse_from_logsum(all);
+  st.tau = threshold_f32(all.m, log_rho);
+  const bool has_a = a >= 0 && a < V;
+  st.z_a = has_a ? Storage<TIn>::widen(row[a]) : 0.f;
+  st.member = has_a && st.z_a >= st.tau;
+  st.e_a = st.member ? ex2((st.z_a - st.m) * kLog2e) : 0.f;
+
+  const int a_part = (has_a && a >= off && a < off + v_part) ? a - off : -1;
+  const SumCount sc = row_sweep2<TIn, kStage>(row + off, v_part, a_part, st.tau, st.m, bound,
+                                              scratch, hot_smem, hot);
+  const SumCount tot = cluster_reduce_sumcount<kCluster>(sc, cl_slots + 4);
   st.s_x = tot.s;
   st.n = tot.n;
 
   // ---- optional packed membership mask (diagnostic output, plain loads)
-  if (mask_row) {
+  if (mask_row && off == 0) {
     const int n_words = (V + 31) / 32;
-    for (int w = tid; w < n_words; w += blockDim.x) {
+    for (int w = threadIdx.x; w < n_words; w += blockDim.x) {
       uint32_t bits = 0;
       for (int b = 0; b < 32; ++b) {
         const long long k = (long long)w * 32 + b;
@@ -397,34 +482,46 @@ __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int
   }
 }
 
-// Shared-memory layout of the row kernel, in 4-byte words.
-__host__ __device__ inline int smem_words_fixed(int threads) { return 96 + (threads / 32) * kHotCap; }
+// Shared-memory layout of the row kernel, in 4-byte words: 96 for the block
+// reductions, 16 for the cluster exchange, then the hot lists, then the bounds.
+__host__ __device__ inline int smem_words_fixed(int threads) {
+  return 96 + 16 + (threads / 32) * kHotCap;
+}
 
 // kThreads / kBlocks: the launch bounds (largest block, blocks per SM) that set
-// the register budget of this instantiation.
-template <typename TIn, typename TGrad, int kStage, int kThreads, int kBlocks>
+// the register budget of this instantiation.  kCluster blocks share one row.
+template <typename TIn, typename TGrad, int kStage, int kThreads, int kBlocks, int kCluster>
 __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowParams p) {
   extern __shared__ __align__(16) float smem[];
-  float *scratch = smem;  // 96 floats for the block reductions
-  uint32_t *hot_smem = reinterpret_cast<uint32_t *>(smem + 96);  // kHotCap per warp
+  float *scratch = smem;        // 96 floats for the block reductions
+  float *cl_slots = smem + 96;  // 4 exchanges x 4 floats, each written once
+  uint32_t *hot_smem = reinterpret_cast<uint32_t *>(smem + 112);  // kHotCap per warp
   uint16_t *bound = reinterpret_cast<uint16_t *>(smem + smem_words_fixed(blockDim.x));
 
-  const long long t = blockIdx.x;
+  constexpr int kElems = Granule<TIn>::kElems;
+  const long long t = blockIdx.x / kCluster;
+  const int rank = kCluster > 1 ? (int)cluster_rank() : 0;
   const long long id = p.ids ? load_id(p.ids, p.id_is_i32, t) : -1;
   const bool has_id = id >= 0, bad_id = id >= p.V;
   const int a = (has_id && !bad_id) ? (int)id : -1;
   const int V = (int)p.V;
+  // this block's part of the row, in whole granules
+  const int n_gran = (V + kElems - 1) / kElems;
+  const int per_rank = (n_gran + kCluster - 1) / kCluster;
+  const int off = min(rank * per_rank, n_gran) * kElems;
+  const int v_part = max(0, min(V - off, per_rank * kElems));
 
   const TIn *trow = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
   uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * ((p.V + 31) / 32) : nullptr;
   HotList hot;
-  const SideStats st =
-      row_stats<TIn, kStage>(trow, V, a, p.log_rho, bound, scratch, hot_smem, hot, mask_t);
+  const SideStats st = row_stats<TIn, kStage, kCluster>(trow, V, off, v_part, a, p.log_rho, bound,
+                                                        scratch, cl_slots, hot_smem, hot, mask_t);
 
   if (p.grad) {
     const float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
-    row_grad<TIn, TGrad, kStage>(trow, reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad, V, a, st,
-                                 g, bound, hot);
+    const int a_part = (a >= off && a < off + v_part) ? a - off : -1;
+    row_grad<TIn, TGrad, kStage>(trow + off, reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad + off,
+                                 v_part, a_part, st, g, bound, hot);
   }
 
   SideStats si;
@@ -433,10 +530,11 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
     const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
     uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
     HotList hot_i;
-    si = row_stats<TIn, kStage>(irow, V, a, p.log_rho, bound, scratch, hot_smem, hot_i, mask_i);
+    si = row_stats<TIn, kStage, kCluster>(irow, V, off, v_part, a, p.log_rho, bound, scratch,
+                                          cl_slots + 8, hot_smem, hot_i, mask_i);
   }
 
-  if (threadIdx.x == 0) {
+  if (threadIdx.x == 0 && rank == 0) {
     const float lt = finish_side(p.out_t, t, st, has_id, bad_id);
     uint8_t flags = (uint8_t)((st.member ? DVP_FLAG_IN_TRAIN : 0) | (has_id ? 0 : DVP_FLAG_NO_ID) |
                               (bad_id ? DVP_FLAG_BAD_ID : 0));
@@ -449,6 +547,8 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
     }
     if (p.flags) p.flags[t] = flags;
   }
+  // no block may leave while another one can still read its exchange slots
+  if constexpr (kCluster > 1) cluster_sync_all();
 }
 
 // ---- scalar kernel: any alignment, any row length ---------------------------
@@ -605,21 +705,37 @@ static inline bool aligned32(const void *base, long long ld, size_t elem) {
   return base == nullptr || (((uintptr_t)base % 32 == 0) && ((ld * (long long)elem) % 32 == 0));
 }
 
-template <typename TIn, typename TGrad, int kStage, int kThreads, int kBlocks>
+template <typename TIn, typename TGrad, int kStage, int kThreads, int kBlocks, int kCluster>
 static cudaError_t launch_rows_vec(const RowParams &p, int threads, size_t smem, cudaStream_t s) {
-  auto k = dvp_row_kernel<TIn, TGrad, kStage, kThreads, kBlocks>;
+  auto k = dvp_row_kernel<TIn, TGrad, kStage, kThreads, kBlocks, kCluster>;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  k<<<(unsigned)p.T, threads, smem, s>>>(p);
-  return cudaGetLastError();
+  if constexpr (kCluster == 1) {
+    k<<<(unsigned)p.T, threads, smem, s>>>(p);
+    return cudaGetLastError();
+  } else {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.T * kCluster), 1, 1);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kCluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k, p);
+  }
 }
 
 template <typename TIn, typename TGrad>
 static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s) {
   constexpr int kElems = Granule<TIn>::kElems;
-  int threads = hint & 0xffff, stage = (hint >> 16) & 0xff;
+  int threads = hint & 0xffff, stage = (hint >> 16) & 0xff, cluster = (hint >> 24) & 0xff;
   // measured on B200: 4-byte logits run best with 2 x 512 threads per SM, 2-byte
   // logits (twice the exponentials per byte) with 4 x 256
   if (threads == 0) threads = sizeof(TIn) == 4 ? 512 : 256;
@@ -627,19 +743,26 @@ static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s
   const bool vec_ok = aligned32(p.train, p.ld_train, sizeof(TIn)) &&
                       aligned32(p.infer, p.ld_infer, sizeof(TIn)) &&
                       aligned32(p.grad, p.ld_grad, sizeof(TGrad));
-  const long long n_gran = (p.V + kElems - 1) / kElems;
+  const long long n_gran_row = (p.V + kElems - 1) / kElems;
+  if (cluster == 0) cluster = 1;
+  if (cluster > 1 && (n_gran_row < 4096 || p.T * cluster > 0x7fffffffLL)) cluster = 1;
+  const long long n_gran = (n_gran_row + cluster - 1) / cluster;  // granules per block
   // shrink the block for short rows so that threads are not idle
   while (threads > 64 && (long long)threads * stage / 2 >= n_gran) threads /= 2;
   const long long per = (long long)stage * threads;
   const size_t smem = (size_t)smem_words_fixed(threads) * 4 +
                       (size_t)((n_gran + per - 1) / per) * per * sizeof(uint16_t);
   if (vec_ok && smem <= 200 * 1024) {
+    if (cluster == 4 && threads <= 256 && stage == 2)
+      return launch_rows_vec<TIn, TGrad, 2, 256, 4, 4>(p, threads, smem, s);
+    if (cluster == 2 && threads <= 256 && stage == 2)
+      return launch_rows_vec<TIn, TGrad, 2, 256, 4, 2>(p, threads, smem, s);
     if (threads > 256) {
-      if (stage == 1) return launch_rows_vec<TIn, TGrad, 1, 512, 2>(p, threads, smem, s);
-      return launch_rows_vec<TIn, TGrad, 2, 512, 2>(p, threads, smem, s);
+      if (stage == 1) return launch_rows_vec<TIn, TGrad, 1, 512, 2, 1>(p, threads, smem, s);
+      return launch_rows_vec<TIn, TGrad, 2, 512, 2, 1>(p, threads, smem, s);
     }
-    if (stage == 1) return launch_rows_vec<TIn, TGrad, 1, 256, 4>(p, threads, smem, s);
-    return launch_rows_vec<TIn, TGrad, 2, 256, 4>(p, threads, smem, s);
+    if (stage == 1) return launch_rows_vec<TIn, TGrad, 1, 256, 4, 1>(p, threads, smem, s);
+    return launch_rows_vec<TIn, TGrad, 2, 256, 4, 1>(p, threads, smem, s);
   }
   dvp_row_kernel_scalar<TIn, TGrad><<<(unsigned)p.T, 512, 0, s>>>(p);
   return cudaGetLastError();

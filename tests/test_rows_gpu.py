@@ -31,21 +31,24 @@ def test_config0_small_fp32_forward_backward():
     assert 1 <= report["mean_safe_set_size"] < 200
 
 
+@pytest.mark.parametrize("cluster", [0, 2, 4])
 @pytest.mark.parametrize("rho", [1e-4, 1e-3])
-def test_bf16_full_vocabulary_rows(rho):
-    """V = 151,936 bf16: several sweeps of a 256-thread block plus a ragged tail."""
+def test_bf16_full_vocabulary_rows(rho, cluster):
+    """V = 151,936 bf16: several sweeps of a 256-thread block plus a ragged tail;
+    one block per row, or a cluster of 2 or 4 blocks sharing each row."""
     w = W["c2_bf16_fwdbwd"]
     batch = inputs.make_rows(w, seed=2, device=DEV, T=96)
-    res = _forward(batch, rho, True)
+    res = _forward(batch, rho, True, launch_hint=(256 | (2 << 16) | (cluster << 24)) if cluster else 0)
     torch.cuda.synchronize()
     report, want = parity.check_forward(res, batch, rho, w.V, True)
     assert report["mean_safe_set_size"] > 5
 
 
-def test_fp32_heavy_tail_262144():
+@pytest.mark.parametrize("cluster", [0, 4])
+def test_fp32_heavy_tail_262144(cluster):
     w = W["c3_f32_heavy"]
     batch = inputs.make_rows(w, seed=3, device=DEV, T=24, chunk_rows=8)
-    res = _forward(batch, 1e-4, True)
+    res = _forward(batch, 1e-4, True, launch_hint=(256 | (2 << 16) | (cluster << 24)) if cluster else 0)
     torch.cuda.synchronize()
     report, want = parity.check_forward(res, batch, 1e-4, w.V, True)
     assert report["mean_safe_set_size"] < 50
