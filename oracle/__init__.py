@@ -288,3 +288,34 @@ def dvp_rows_f64(z: np.ndarray, ids: np.ndarray, rho: float, upstream: np.ndarra
             lib.dvp_oracle_side_grad(z.ctypes.data + t * V * 8, V, int(ids[t]), float(upstream[t]), p,
                                      grad.ctypes.data + t * V * 8)
     return Result(train=_side(side, mask), infer=None, log_ratio=None, grad=grad)
+
+
+@dataclass
+class SequenceResult:
+    seq_log_ratio: np.ndarray   # [S] Delta_y = sum of the token log-ratios
+    min_log_ratio: np.ndarray   # [S]
+    n_valid: np.ndarray         # [S] tokens with a sampled id
+    n_zero_weight: np.ndarray   # [S] tokens outside the training safe set
+    veto: np.ndarray            # [S] 1 when some token weight is below the threshold
+
+
+def dvp_sequences(log_ratio: np.ndarray, seq_offsets: np.ndarray, veto_threshold: float = 1e-4
+                  ) -> SequenceResult:
+    """Sequence-level mismatch and token veto (Sec. 4.4, Thm. 5.3, App. A protocol 5)."""
+    lib = _load()
+    lr = np.ascontiguousarray(log_ratio, dtype=np.float64)
+    off = np.ascontiguousarray(seq_offsets, dtype=np.int64)
+    S = len(off) - 1
+    assert S >= 0 and (S == 0 or (off[0] >= 0 and off[-1] <= len(lr) and (np.diff(off) >= 0).all()))
+    out = SequenceResult(np.zeros(S), np.zeros(S), np.zeros(S, dtype=np.int64),
+                         np.zeros(S, dtype=np.int64), np.zeros(S, dtype=np.uint8))
+    lib.dvp_oracle_sequences.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_double,
+                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                         ctypes.c_void_p, ctypes.c_void_p]
+    lib.dvp_oracle_sequences.restype = None
+    if S > 0:
+        lib.dvp_oracle_sequences(lr.ctypes.data, off.ctypes.data, S, float(veto_threshold),
+                                 out.seq_log_ratio.ctypes.data, out.min_log_ratio.ctypes.data,
+                                 out.n_valid.ctypes.data, out.n_zero_weight.ctypes.data,
+                                 out.veto.ctypes.data)
+    return out

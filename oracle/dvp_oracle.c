@@ -260,5 +260,42 @@ int dvp_oracle_batch(const oracle_batch *b, int nthreads) {
   return nthreads;
 }
 
+/*
+ * Sequence level (Sec. 4.4: Delta_y = sum_t Delta_{a_t}; Thm. 5.3: the ratio of a
+ * trajectory is the product of its token ratios; App. A protocol 5: a token whose
+ * importance weight pi^mp_train / pi^mp_infer falls below the veto threshold
+ * discards the whole sequence).  Tokens of sequence s are [off[s], off[s+1]).
+ * A token without a sampled id (NaN log-ratio) is skipped.  A token outside the
+ * training safe set has weight zero: the sequence sum is -inf whatever else it
+ * holds, and the sequence is vetoed for any positive threshold.
+ */
+void dvp_oracle_sequences(const double *log_ratio, const int64_t *off, int64_t S,
+                          double veto_threshold, double *seq_log_ratio, double *min_log_ratio,
+                          int64_t *n_valid, int64_t *n_zero_weight, uint8_t *veto) {
+  for (int64_t s = 0; s < S; ++s) {
+    nsum acc = {0, 0};
+    double lo = INFINITY;
+    int64_t valid = 0, zero = 0;
+    int has_pinf = 0, vetoed = 0;
+    for (int64_t t = off[s]; t < off[s + 1]; ++t) {
+      const double r = log_ratio[t];
+      if (isnan(r)) continue;
+      ++valid;
+      if (r < lo) lo = r;
+      if (exp(r) < veto_threshold) vetoed = 1;
+      if (isinf(r)) {
+        if (r < 0) ++zero; else has_pinf = 1;
+      } else {
+        nsum_add(&acc, r);
+      }
+    }
+    seq_log_ratio[s] = zero ? -INFINITY : (has_pinf ? INFINITY : nsum_value(&acc));
+    min_log_ratio[s] = lo;
+    n_valid[s] = valid;
+    n_zero_weight[s] = zero;
+    veto[s] = (uint8_t)vetoed;
+  }
+}
+
 int dvp_oracle_sizeof_side(void) { return (int)sizeof(oracle_side); }
 int dvp_oracle_sizeof_batch(void) { return (int)sizeof(oracle_batch); }

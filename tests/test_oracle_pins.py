@@ -249,7 +249,7 @@ def test_log_ratio_sign_and_conventions():
 def test_printed_constants():
     with open(os.path.join(GOLDEN, "paper_constants.txt")) as f:
         rows = [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
-    assert len(rows) == 3
+    assert len(rows) == 4
     for name, expr, printed, digits, *_ in rows:
         value = eval(expr, {"exp": math.exp})
         assert float(f"{value:.{int(digits) - 1}e}") == float(printed), name
@@ -320,3 +320,39 @@ def test_fused_lmhead_matches_autograd_through_the_head():
     # infer side: an ordinary row pass on the stored bf16 logits
     ref_i = oracle.dvp_rows(bits(zi), ids, rho, dtype=oracle.BF16)
     assert np.array_equal(res.rows.infer.logp_mp, ref_i.train.logp_mp)
+
+
+def test_sequence_level_ratio_is_the_product_of_token_ratios_and_veto_rule():
+    """Sec. 4.4 (Delta_y = sum of token mismatches), Thm. 5.3 (trajectory ratio =
+    product of token ratios), App. A protocol 5 (veto below 1e-4)."""
+    rng = np.random.default_rng(31)
+    T, V = 60, 50
+    z = _rows(rng, T, V, scale=2.0)
+    zi = z + rng.normal(size=z.shape) * 0.05
+    ids = rng.integers(0, V, size=T)
+    tr = oracle.dvp_rows_f64(z, ids, 1e-2).train
+    inf = oracle.dvp_rows_f64(zi, ids, 1e-2).train
+    lr = np.where(tr.member == 0, -np.inf, np.where(inf.member == 0, np.inf, tr.logp_mp - inf.logp_mp))
+    off = np.array([0, 7, 7, 30, 60])                       # one empty sequence
+    res = oracle.dvp_sequences(lr, off, 1e-4)
+    with open(os.path.join(GOLDEN, "paper_constants.txt")) as f:
+        veto_printed = [float(ln.split()[2]) for ln in f if ln.startswith("veto_threshold")][0]
+    for s in range(4):
+        seg = slice(off[s], off[s + 1])
+        w = np.where(tr.member[seg] == 0, 0.0, np.exp(lr[seg]))       # token weights pi^mp_t / pi^mp_i
+        prod = np.prod(w)
+        if res.n_zero_weight[s] == 0 and np.isfinite(res.seq_log_ratio[s]):
+            assert math.exp(res.seq_log_ratio[s]) == pytest.approx(prod, rel=1e-12)
+            both = (tr.member[seg] == 1) & (inf.member[seg] == 1)
+            direct = math.fsum(tr.logp_mp[seg][both]) - math.fsum(inf.logp_mp[seg][both])
+            assert res.seq_log_ratio[s] == pytest.approx(direct, abs=1e-12)
+        elif res.n_zero_weight[s] > 0:
+            assert prod == 0.0 and res.seq_log_ratio[s] == -np.inf
+        assert res.veto[s] == int((w < veto_printed).any())
+        assert res.n_valid[s] == off[s + 1] - off[s]
+        assert res.n_zero_weight[s] == int((tr.member[seg] == 0).sum())
+    assert res.seq_log_ratio[1] == 0.0 and res.veto[1] == 0 and res.min_log_ratio[1] == np.inf
+    # the veto threshold acts on the weight, not on its logarithm
+    res = oracle.dvp_sequences(np.array([0.0, math.log(1.01e-4), 0.1, math.log(0.99e-4), np.nan]),
+                               np.array([0, 3, 5]), 1e-4)
+    assert res.veto.tolist() == [0, 1] and res.n_valid.tolist() == [3, 1]
