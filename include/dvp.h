@@ -229,6 +229,46 @@ typedef struct {
 int dvp_fused_lmhead_forward_backward(const dvp_fused_args *args);
 
 /*
+ * dvp_sequence_aggregate -- sequence-level view of the per-token results: the
+ * mismatch of a trajectory is the sum of its token mismatches (Sec. 4.4,
+ * Delta_y = sum_t Delta_{a_t}), its importance ratio the product of the token
+ * ratios (Thm. 5.3), and a token whose importance weight
+ * pi^mp_train / pi^mp_infer = exp(log_ratio) is below `veto_threshold` marks
+ * the whole sequence as discarded (App. A, protocol 5; the paper uses 1e-4).
+ *
+ *   seq_offsets    device [S + 1] int64, non-decreasing; sequence s owns tokens
+ *                  [seq_offsets[s], seq_offsets[s+1]), all within [0, T)
+ *   log_ratio      device [T] float32 as written by dvp_forward: NaN = token
+ *                  without a sampled id (skipped), -inf = outside the training
+ *                  safe set (weight zero), +inf = outside the inference set only
+ *   seq_log_ratio  device [S]: sum of the token log-ratios; -inf if any token
+ *                  has weight zero, else +inf if any token is +inf
+ *   min_log_ratio  device [S]: smallest token log-ratio (+inf for an empty sequence)
+ *   n_valid        device [S] int32: tokens with a sampled id
+ *   n_zero_weight  device [S] int32: tokens with weight zero
+ *   veto           device [S] bytes: 1 when some token weight < veto_threshold
+ * Each output may be NULL.  veto_threshold >= 0 (0 never vetoes).  S = 0 is a
+ * no-op.  Errors: DVP_ERR_INVALID_ARG (null inputs, negative sizes, negative or
+ * NaN threshold).  Offsets are not checked on the device.
+ */
+typedef struct {
+  uint32_t struct_size;
+  uint32_t reserved_;
+  int64_t T, S;
+  const int64_t *seq_offsets;
+  const float *log_ratio;
+  double veto_threshold;
+  float *seq_log_ratio;
+  float *min_log_ratio;
+  int32_t *n_valid;
+  int32_t *n_zero_weight;
+  uint8_t *veto;
+  void *stream;
+} dvp_sequence_args;
+
+int dvp_sequence_aggregate(const dvp_sequence_args *args);
+
+/*
  * dvp_fused_lmhead_forward_backward_static -- the fused entry point for callers
  * that cannot obtain device memory of their own.  (The paper has no counterpart;
  * this is a packaging variant of the entry point above.)

@@ -24,7 +24,7 @@ DVP_ENTRY_FORWARD, DVP_ENTRY_BACKWARD, DVP_ENTRY_FUSED_LMHEAD = 0, 1, 2
 DVP_STATIC_WORKSPACE_BYTES = 32 * 1024 * 1024
 
 EXPORTS = ("dvp_forward", "dvp_backward", "dvp_fused_lmhead_forward_backward",
-           "dvp_fused_lmhead_forward_backward_static", "dvp_gemm_tn",
+           "dvp_fused_lmhead_forward_backward_static", "dvp_sequence_aggregate", "dvp_gemm_tn",
            "dvp_workspace_bytes", "dvp_status_string", "dvp_version")
 
 _DTYPES = {torch.float32: DVP_F32, torch.bfloat16: DVP_BF16, torch.float16: DVP_F16}
@@ -125,6 +125,24 @@ class FusedArgs(ctypes.Structure):
     ]
 
 
+class SequenceArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("reserved_", ctypes.c_uint32),
+        ("T", ctypes.c_int64),
+        ("S", ctypes.c_int64),
+        ("seq_offsets", ctypes.c_void_p),
+        ("log_ratio", ctypes.c_void_p),
+        ("veto_threshold", ctypes.c_double),
+        ("seq_log_ratio", ctypes.c_void_p),
+        ("min_log_ratio", ctypes.c_void_p),
+        ("n_valid", ctypes.c_void_p),
+        ("n_zero_weight", ctypes.c_void_p),
+        ("veto", ctypes.c_void_p),
+        ("stream", ctypes.c_void_p),
+    ]
+
+
 _lib = None
 
 
@@ -145,6 +163,8 @@ def load_library() -> ctypes.CDLL:
         lib.dvp_fused_lmhead_forward_backward.restype = ctypes.c_int
         lib.dvp_fused_lmhead_forward_backward_static.argtypes = [ctypes.POINTER(FusedArgs)]
         lib.dvp_fused_lmhead_forward_backward_static.restype = ctypes.c_int
+        lib.dvp_sequence_aggregate.argtypes = [ctypes.POINTER(SequenceArgs)]
+        lib.dvp_sequence_aggregate.restype = ctypes.c_int
         lib.dvp_gemm_tn.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64,
                                     ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int64, ctypes.c_int32, ctypes.c_float, ctypes.c_int32,
@@ -424,4 +444,34 @@ def dvp_fused_lmhead_forward_backward_static(hidden: torch.Tensor, w_vocab: torc
     st = lib.dvp_fused_lmhead_forward_backward_static(ctypes.byref(a))
     if st != DVP_OK:
         raise DvpError(st, "dvp_fused_lmhead_forward_backward_static")
+    return res
+
+
+def dvp_sequence_aggregate(log_ratio: torch.Tensor, seq_offsets: torch.Tensor,
+                           veto_threshold: float = 1e-4, stream=None):
+    """Per-sequence sum and minimum of the token log-ratios, token counts and the
+    veto flag (Sec. 4.4, Thm. 5.3, App. A protocol 5).  ``seq_offsets`` is an
+    int64 device tensor of S + 1 non-decreasing token offsets."""
+    lib = load_library()
+    if log_ratio.dtype != torch.float32 or seq_offsets.dtype != torch.int64:
+        raise TypeError("log_ratio must be float32 and seq_offsets int64")
+    S = seq_offsets.numel() - 1
+    dev = log_ratio.device
+    res = SimpleNamespace(
+        seq_log_ratio=torch.empty(S, dtype=torch.float32, device=dev),
+        min_log_ratio=torch.empty(S, dtype=torch.float32, device=dev),
+        n_valid=torch.empty(S, dtype=torch.int32, device=dev),
+        n_zero_weight=torch.empty(S, dtype=torch.int32, device=dev),
+        veto=torch.empty(S, dtype=torch.uint8, device=dev))
+    a = SequenceArgs()
+    a.struct_size = ctypes.sizeof(SequenceArgs)
+    a.T, a.S = log_ratio.numel(), S
+    a.seq_offsets, a.log_ratio = _ptr(seq_offsets), _ptr(log_ratio)
+    a.veto_threshold = float(veto_threshold)
+    a.seq_log_ratio, a.min_log_ratio = _ptr(res.seq_log_ratio), _ptr(res.min_log_ratio)
+    a.n_valid, a.n_zero_weight, a.veto = _ptr(res.n_valid), _ptr(res.n_zero_weight), _ptr(res.veto)
+    a.stream = _stream(stream)
+    st = lib.dvp_sequence_aggregate(ctypes.byref(a))
+    if st != DVP_OK:
+        raise DvpError(st, "dvp_sequence_aggregate")
     return res

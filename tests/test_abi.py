@@ -37,7 +37,8 @@ def test_every_declared_symbol_is_exported(lib):
 def test_struct_layout_matches_the_header(tmp_path):
     from paper_2512_23087_b200 import binding
     structs = {"dvp_forward_args": binding.ForwardArgs, "dvp_backward_args": binding.BackwardArgs,
-               "dvp_fused_args": binding.FusedArgs, "dvp_side_out": binding.SideOut}
+               "dvp_fused_args": binding.FusedArgs, "dvp_side_out": binding.SideOut,
+               "dvp_sequence_args": binding.SequenceArgs}
     lines = []
     for cname, cls in structs.items():
         lines.append(f'printf("{cname} %zu\\n", sizeof({cname}));')
@@ -104,6 +105,17 @@ def test_argument_errors_are_reported_before_any_launch(lib):
     assert lib.dvp_backward(ctypes.byref(bw)) == b.DVP_ERR_INVALID_ARG        # missing pointers
     fa = b.FusedArgs()
     assert lib.dvp_fused_lmhead_forward_backward(ctypes.byref(fa)) == b.DVP_ERR_INVALID_ARG
+    assert lib.dvp_fused_lmhead_forward_backward_static(ctypes.byref(fa)) == b.DVP_ERR_INVALID_ARG
+    sa = b.SequenceArgs()
+    sa.struct_size = ctypes.sizeof(b.SequenceArgs)
+    sa.S, sa.T = 3, 10
+    assert lib.dvp_sequence_aggregate(ctypes.byref(sa)) == b.DVP_ERR_INVALID_ARG   # null inputs
+    sa.veto_threshold = -1.0
+    sa.seq_offsets, sa.log_ratio = 0x1000, 0x2000
+    assert lib.dvp_sequence_aggregate(ctypes.byref(sa)) == b.DVP_ERR_INVALID_ARG   # negative threshold
+    sa.S = 0
+    sa.veto_threshold = 1e-4
+    assert lib.dvp_sequence_aggregate(ctypes.byref(sa)) == b.DVP_OK                # no sequences: no-op
 
 
 def test_missing_library_fails_loudly(tmp_path, monkeypatch):

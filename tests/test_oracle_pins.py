@@ -332,7 +332,8 @@ def test_sequence_level_ratio_is_the_product_of_token_ratios_and_veto_rule():
     ids = rng.integers(0, V, size=T)
     tr = oracle.dvp_rows_f64(z, ids, 1e-2).train
     inf = oracle.dvp_rows_f64(zi, ids, 1e-2).train
-    lr = np.where(tr.member == 0, -np.inf, np.where(inf.member == 0, np.inf, tr.logp_mp - inf.logp_mp))
+    with np.errstate(invalid="ignore"):
+        lr = np.where(tr.member == 0, -np.inf, np.where(inf.member == 0, np.inf, tr.logp_mp - inf.logp_mp))
     off = np.array([0, 7, 7, 30, 60])                       # one empty sequence
     res = oracle.dvp_sequences(lr, off, 1e-4)
     with open(os.path.join(GOLDEN, "paper_constants.txt")) as f:
