@@ -253,6 +253,27 @@ def run_ours(args):
     clocks = sampler.stop()
     launches = args.steps          # one kernel per dvp_forward call
 
+    # the workload's other threshold, timed the same way and reported beside the headline
+    other = None
+    if args.rho is None and len(w.rhos) > 1:
+        rho2 = w.rhos[1]
+        res2 = None
+        for _ in range(3):
+            res2 = binding.dvp_forward(batch.train, batch.ids, rho2, infer_logits=batch.infer,
+                                       upstream=batch.upstream if w.backward else None,
+                                       grad_dtype=grad_dtype, stream=stream, out=res2)
+        barrier()
+        ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev2.record(stream)
+        for _ in range(args.steps):
+            binding.dvp_forward(batch.train, batch.ids, rho2, infer_logits=batch.infer,
+                                upstream=batch.upstream if w.backward else None,
+                                grad_dtype=grad_dtype, stream=stream, out=res2)
+        ev3.record(stream)
+        barrier()
+        other = {"rho": rho2, "ms_per_step": ev2.elapsed_time(ev3) / args.steps}
+        launches += args.steps
+
     # ---- end to end: host buffers in, per-token results out, copies inside the timed region
     slab = min(T, 2048)
     n_slabs = (T + slab - 1) // slab
@@ -345,6 +366,15 @@ def run_ours(args):
                      "kernel": "dvp_row_kernel", "bytes_per_launch": alg_bytes,
                      "frac_of_nominal_8TBs": achieved / 8000.0},
     }
+    if other is not None:
+        if world > 1:
+            t2 = torch.tensor([other["ms_per_step"]], device=dev, dtype=torch.float64)
+            torch.distributed.all_reduce(t2, op=torch.distributed.ReduceOp.MAX)
+            other["ms_per_step"] = t2.item()
+        sec2 = other["ms_per_step"] * 1e-3
+        other.update(value=tokens / sec2, unit=UNIT, achieved_gbs=alg_bytes / sec2 / 1e9,
+                     frac=alg_bytes / sec2 / 1e9 / peak)
+        line["other_threshold"] = other
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(batch, rho, w.backward)

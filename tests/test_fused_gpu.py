@@ -178,3 +178,30 @@ def test_fused_argument_errors():
         binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, 1e-3,
                                                   batch.upstream, workspace=torch.empty(512, dtype=torch.uint8, device=DEV))
     assert e.value.status == binding.DVP_ERR_WORKSPACE
+
+
+def test_fused_missing_and_out_of_range_ids_and_empty_batch():
+    w = inputs.WORKLOADS["c4_fused_lmhead"]
+    batch = inputs.make_fused(w, seed=2, device=DEV, T=40, H=128, V=1024)
+    batch.ids[3] = -1
+    batch.ids[7] = 5000
+    res = binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, 1e-2,
+                                                    batch.upstream, infer_logits=batch.infer)
+    torch.cuda.synchronize()
+    flags = res.flags.tolist()
+    assert flags[3] & binding.DVP_FLAG_NO_ID and flags[7] & binding.DVP_FLAG_BAD_ID
+    assert torch.isnan(res.train.logp_mp[[3, 7]]).all() and torch.isnan(res.log_ratio[[3, 7]]).all()
+    assert res.d_hidden[[3, 7]].abs().max().item() == 0.0
+    ids = batch.ids.clone()
+    ids[3] = 0
+    ids[7] = 0
+    want = oracle.dvp_fused_lmhead(_bits(batch.hidden), _bits(batch.w_vocab), _bits(batch.infer),
+                                   batch.ids.cpu().numpy(), 1e-2, batch.upstream.cpu().numpy().astype(np.float64))
+    keep = np.ones(40, dtype=bool)
+    keep[[3, 7]] = False
+    num = np.linalg.norm(res.d_hidden.cpu().double().numpy()[keep] - want.d_hidden[keep], axis=1)
+    den = np.linalg.norm(want.d_hidden[keep], axis=1)
+    assert (num <= 1e-3 * den + 1e-6 * den.max()).all()
+    empty = binding.dvp_fused_lmhead_forward_backward(batch.hidden[:0], batch.w_vocab, batch.ids[:0], 1e-2,
+                                                      batch.upstream[:0])
+    assert empty.d_hidden.shape[0] == 0
