@@ -317,6 +317,9 @@ int dvp_fused_lmhead_forward_backward_static(const dvp_fused_args *args);
  * row-major, fp32 accumulation.  The paper has no counterpart; it is the
  * "hidden x W_vocab" product of the LM head and its two transposes.
  *   a, b, c   device; lda, ldb, ldc multiples of 8; a, b 16-byte, c 32-byte aligned
+ *   accumulate  bit 0: add to C instead of overwriting it; bit 1: use the kernel that
+ *             gives each 128 x 256 tile to one block instead of 256 x 256 tiles to
+ *             pairs of blocks (same results up to summation order; for comparison)
  *   status    device int32, written non-zero if a kernel gave up waiting
  * Errors: DVP_ERR_INVALID_ARG (null pointers, negative sizes),
  * DVP_ERR_UNSUPPORTED (dtype, alignment), DVP_ERR_CUDA.

@@ -315,7 +315,7 @@ def dvp_backward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, upst
 
 
 def dvp_gemm_tn(a: torch.Tensor, b: torch.Tensor, *, alpha: float = 1.0, out: torch.Tensor | None = None,
-                accumulate: bool = False, stream=None):
+                accumulate: bool = False, single_block_tiles: bool = False, stream=None):
     """``out (+)= alpha * a @ b.T`` on the tensor cores; a [m, k] and b [n, k] are
     both bf16 or both f16 with k contiguous, out is float32.  Returns (out, status)
     where status is a device int32 that is non-zero if the kernel gave up waiting."""
@@ -330,7 +330,8 @@ def dvp_gemm_tn(a: torch.Tensor, b: torch.Tensor, *, alpha: float = 1.0, out: to
         out = torch.empty(m, n, dtype=torch.float32, device=a.device)
     status = torch.zeros(1, dtype=torch.int32, device=a.device)
     st = lib.dvp_gemm_tn(_ptr(a), a.stride(0), _ptr(b), b.stride(0), _ptr(out), out.stride(0), m, n, k,
-                         _DTYPES[a.dtype], float(alpha), int(accumulate), _ptr(status), _stream(stream))
+                         _DTYPES[a.dtype], float(alpha), int(accumulate) | (2 if single_block_tiles else 0),
+                         _ptr(status), _stream(stream))
     if st != DVP_OK:
         raise DvpError(st, "dvp_gemm_tn")
     return out, status

@@ -200,7 +200,8 @@ int dvp_gemm_tn(const void *a, int64_t lda, const void *b, int64_t ldb, float *c
     return DVP_ERR_CUDA;
   const cudaError_t e =
       dvp::gemm::launch_gemm_tn(a, lda, b, ldb, c, ldc, (int)m, (int)n, (int)k, dtype == DVP_BF16, alpha,
-                                nullptr, accumulate != 0, status, sms, static_cast<cudaStream_t>(stream));
+                                nullptr, (accumulate & 1) != 0, status, sms,
+                                static_cast<cudaStream_t>(stream), (accumulate & 2) != 0);
   if (e == cudaErrorInvalidValue) return DVP_ERR_UNSUPPORTED;
   return e == cudaSuccess ? DVP_OK : DVP_ERR_CUDA;
 }

@@ -319,6 +319,245 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   }
 }
 
+// ---- the same contraction on pairs of blocks (tcgen05 cta_group::2) ------------------
+// Two blocks of a cluster share one 256 x 256 output tile: each holds 128 rows of
+// A, 128 of the 256 rows of B, and the 128 x 256 accumulator of its own rows in its
+// tensor memory.  One thread of the leader block (cluster rank 0) issues the MMAs for
+// both, so each block reads only half of B from shared memory per MMA: this removes
+// the shared-memory bandwidth ceiling of the one-block form.  Both blocks' TMA loads
+// complete on the leader's "full" barrier; the MMA thread's commits arrive on the
+// "empty" and "accumulator full" barriers of both blocks; both blocks' epilogue warps
+// arrive on the leader's "accumulator empty" barrier.
+
+constexpr int kPairBM = 256;
+constexpr int kStages2 = 6;
+constexpr uint32_t kBytesB2 = (kBN / 2) * kBK * 2;
+constexpr uint32_t kStageBytes2 = kBytesA + kBytesB2;
+constexpr size_t kSmemBytes2 = 1024 + (size_t)kStages2 * kStageBytes2 + 256;
+
+struct Shared2 {
+  uint64_t full[kStages2], empty[kStages2], tmem_full[2], tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of this block's shared-memory location `local` as seen in block `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr)
+               : "memory");
+}
+// TMA tile load whose completion is counted on a barrier that may live in the peer block.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map,
+                                                 uint32_t bar_cluster_addr, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], "
+      "[%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void umma_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrive, once these MMAs are done, on the barrier at this offset in both blocks of the pair.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], "
+      "%1;" ::"r"(bar),
+      "h"(mask)
+      : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                    const Params p, const uint32_t fmt) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *aligned = smem_raw + (base - smem_u32(smem_raw));
+  Shared2 *sh = reinterpret_cast<Shared2 *>(aligned + (size_t)kStages2 * kStageBytes2);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();  // 0 = leader of the pair
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  const int tiles_m = (p.M + kPairBM - 1) / kPairBM, tiles_n = (p.N + kBN - 1) / kBN;
+  const int n_tiles = tiles_m * tiles_n;
+  const int k_slices = (p.K + kBK - 1) / kBK;
+  const bool m_fastest = tiles_m <= tiles_n;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages2; ++s) {
+      mbar_init(smem_u32(&sh->full[s]), 1);   // the leader's producer, plus the bytes of both blocks
+      mbar_init(smem_u32(&sh->empty[s]), 1);  // one commit
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&sh->tmem_full[b]), 1);   // one commit
+      mbar_init(smem_u32(&sh->tmem_empty[b]), 8);  // four epilogue warps in each block
+    }
+    sh->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(&sh->tmem_base)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  cluster_barrier();  // barriers of both blocks are initialised before anyone signals them
+  tc_fence_after();
+  const uint32_t tmem_base = sh->tmem_base;
+  volatile int *abort_flag = &sh->abort_flag;
+
+  if (warp == 0) {
+    // ---------------- producer (both blocks): own rows of A, own half of B
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int tile = pair; tile < n_tiles && !*abort_flag; tile += n_pairs) {
+        const int tm = m_fastest ? tile % tiles_m : tile / tiles_n;
+        const int tn = m_fastest ? tile / tiles_m : tile % tiles_n;
+        for (int ks = 0; ks < k_slices; ++ks, ++it) {
+          const uint32_t s = it % kStages2, round = it / kStages2;
+          if (round > 0 && !mbar_wait(smem_u32(&sh->empty[s]), (round - 1) & 1, abort_flag)) {
+            if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, kErrProducerWait); }
+            break;
+          }
+          const uint32_t bar_local = smem_u32(&sh->full[s]);
+          if (rank == 0) mbar_expect_tx(bar_local, 2 * kStageBytes2);
+          const uint32_t bar = map_to_rank(bar_local, 0);
+          const uint32_t dst = base + s * kStageBytes2;
+          tma_load_2d_pair(dst, &map_a, bar, ks * kBK, tm * kPairBM + (int)rank * kBM);
+          tma_load_2d_pair(dst + kBytesA, &map_b, bar, ks * kBK, tn * kBN + (int)rank * (kBN / 2));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (leader block only)
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kBN >> 3) << 17) |
+                             ((uint32_t)(kPairBM >> 4) << 24);
+      uint32_t it = 0, local_tile = 0;
+      for (int tile = pair; tile < n_tiles && !*abort_flag; tile += n_pairs, ++local_tile) {
+        const uint32_t buf = local_tile & 1, use = local_tile >> 1;
+        if (use > 0 && !mbar_wait(smem_u32(&sh->tmem_empty[buf]), (use - 1) & 1, abort_flag)) {
+          if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, kErrMmaWaitTmem); }
+          break;
+        }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + buf * kBN;
+        bool ok = true;
+        for (int ks = 0; ks < k_slices; ++ks, ++it) {
+          const uint32_t s = it % kStages2, round = it / kStages2;
+          if (!mbar_wait(smem_u32(&sh->full[s]), round & 1, abort_flag)) {
+            if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, kErrMmaWaitFull); }
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t a_addr = base + s * kStageBytes2, b_addr = a_addr + kBytesA;
+          const uint64_t adesc = smem_desc_sw128(a_addr), bdesc = smem_desc_sw128(b_addr);
+#pragma unroll
+          for (int k = 0; k < kBK / kUmmaK; ++k) {
+            const uint64_t step = (uint64_t)((k * kUmmaK * 2) >> 4);
+            umma_pair(tmem_d, adesc + step, bdesc + step, idesc, (ks > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit_pair(smem_u32(&sh->empty[s]));
+        }
+        if (!ok) break;
+        umma_commit_pair(smem_u32(&sh->tmem_full[buf]));
+      }
+    }
+  } else {
+    // ---------------- epilogue (both blocks): own 128 rows of the pair's tile
+    const int quarter = warp & 3;
+    const float alpha = p.alpha * (p.alpha_dev ? *p.alpha_dev : 1.f);
+    uint32_t local_tile = 0;
+    for (int tile = pair; tile < n_tiles && !*abort_flag; tile += n_pairs, ++local_tile) {
+      const int tm = m_fastest ? tile % tiles_m : tile / tiles_n;
+      const int tn = m_fastest ? tile / tiles_m : tile % tiles_n;
+      const uint32_t buf = local_tile & 1, use = local_tile >> 1;
+      if (!mbar_wait(smem_u32(&sh->tmem_full[buf]), use & 1, abort_flag)) {
+        if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, kErrEpilogueWait); }
+        break;
+      }
+      tc_fence_after();
+      const int row = tm * kPairBM + (int)rank * kBM + quarter * 32 + lane;
+      float *crow = p.C + (long long)row * p.ldc;
+#pragma unroll 1
+      for (int c0 = 0; c0 < kBN; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kBN + c0, r);
+        tmem_wait_ld();
+        const int col = tn * kBN + c0;
+        if (row < p.M && col < p.N) {
+          if (col + 32 <= p.N) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              uint32_t w[8];
+              if (p.accumulate) {
+                const float4 o0 = *reinterpret_cast<const float4 *>(crow + col + j);
+                const float4 o1 = *reinterpret_cast<const float4 *>(crow + col + j + 4);
+                const float old[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                  w[e] = __float_as_uint(fmaf(alpha, __uint_as_float(r[j + e]), old[e]));
+              } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) w[e] = __float_as_uint(alpha * __uint_as_float(r[j + e]));
+              }
+              asm volatile("st.global.v8.u32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(crow + col + j),
+                           "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]),
+                           "r"(w[7])
+                           : "memory");
+            }
+          } else {
+            for (int j = 0; j < 32 && col + j < p.N; ++j) {
+              const float v = alpha * __uint_as_float(r[j]);
+              crow[col + j] = p.accumulate ? crow[col + j] + v : v;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote(map_to_rank(smem_u32(&sh->tmem_empty[buf]), 0));
+    }
+  }
+
+  // ---------------- teardown: nobody frees tensor memory the pair still uses
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(500);
+  }
+  cluster_barrier();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols)
+                 : "memory");
+  }
+}
+
 // ---- host side ------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
@@ -361,17 +600,41 @@ inline bool make_map(CUtensorMap *map, const void *base, long long rows, long lo
 inline cudaError_t launch_gemm_tn(const void *A, long long lda, const void *B, long long ldb, float *C,
                                   long long ldc, int M, int N, int K, bool is_bf16, float alpha,
                                   const float *alpha_dev, bool accumulate, int *status, int sm_count,
-                                  cudaStream_t stream) {
+                                  cudaStream_t stream, bool single_block_tiles = false) {
   if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
   if (lda % 8 || ldb % 8 || ldc % 8 || (uintptr_t)A % 16 || (uintptr_t)B % 16 || (uintptr_t)C % 32)
     return cudaErrorInvalidValue;
+  Params p{C, ldc, M, N, K, alpha, alpha_dev, accumulate ? 1 : 0, status};
   CUtensorMap map_a, map_b;
+  if (!single_block_tiles) {
+    // pairs of blocks on 256 x 256 tiles
+    if (!make_map(&map_a, A, M, K, lda, kBM, is_bf16) || !make_map(&map_b, B, N, K, ldb, kBN / 2, is_bf16))
+      return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(gemm_tn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kSmemBytes2);
+    if (e != cudaSuccess) return e;
+    const int tiles = ((M + kPairBM - 1) / kPairBM) * ((N + kBN - 1) / kBN);
+    int pairs = sm_count / 2;
+    if (pairs > tiles) pairs = tiles;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = kSmemBytes2;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_tn_pair_kernel, map_a, map_b, p, is_bf16 ? 1u : 0u);
+  }
   if (!make_map(&map_a, A, M, K, lda, kBM, is_bf16) || !make_map(&map_b, B, N, K, ldb, kBN, is_bf16))
     return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(gemm_tn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)kSmemBytes);
   if (e != cudaSuccess) return e;
-  Params p{C, ldc, M, N, K, alpha, alpha_dev, accumulate ? 1 : 0, status};
   const int tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
   const int grid = tiles < sm_count ? tiles : sm_count;
   gemm_tn_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, p, is_bf16 ? 1u : 0u);

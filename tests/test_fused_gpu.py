@@ -29,15 +29,17 @@ def _bits(x):
     return x.detach().cpu().view(torch.int16).numpy().view(np.uint16)
 
 
+@pytest.mark.parametrize("single", [False, True])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
 @pytest.mark.parametrize("m,n,k", [(128, 256, 64), (128, 256, 512), (300, 520, 200), (1, 8, 8),
                                    (1000, 776, 1032), (257, 4096, 4104), (2048, 512, 8192)])
-def test_gemm_tn_matches_float64_matmul(dtype, m, n, k):
+def test_gemm_tn_matches_float64_matmul(dtype, m, n, k, single):
+    """Both kernels: 256 x 256 tiles on pairs of blocks (default) and 128 x 256 tiles on single blocks."""
     g = torch.Generator(device=DEV).manual_seed(m * 7 + n * 3 + k)
     a = torch.randn(m, k, generator=g, device=DEV).to(dtype)
     b = torch.randn(n, k, generator=g, device=DEV).to(dtype)
     ref = (a.double() @ b.double().t())
-    out, status = binding.dvp_gemm_tn(a, b, alpha=0.5)
+    out, status = binding.dvp_gemm_tn(a, b, alpha=0.5, single_block_tiles=single)
     torch.cuda.synchronize()
     assert status.item() == 0
     # fp32 accumulation in tensor memory: up to one unit in the last place per 16-wide step
@@ -45,7 +47,8 @@ def test_gemm_tn_matches_float64_matmul(dtype, m, n, k):
     err = (out.double() - 0.5 * ref).abs().max().item()
     assert err <= tol, (err, tol)
     # accumulate on top, strided operands, misaligned-free views
-    out2, status = binding.dvp_gemm_tn(a, b, alpha=0.25, out=out.clone(), accumulate=True)
+    out2, status = binding.dvp_gemm_tn(a, b, alpha=0.25, out=out.clone(), accumulate=True,
+                                       single_block_tiles=single)
     torch.cuda.synchronize()
     assert status.item() == 0
     assert (out2.double() - 0.75 * ref).abs().max().item() <= 2 * tol
