@@ -319,3 +319,53 @@ def dvp_sequences(log_ratio: np.ndarray, seq_offsets: np.ndarray, veto_threshold
                                  out.n_valid.ctypes.data, out.n_zero_weight.ctypes.data,
                                  out.veto.ctypes.data)
     return out
+
+
+_LISTING_DTYPE = np.dtype([("max", "f8"), ("lse_full", "f8"), ("lse_masked", "f8"), ("logp_masked", "f8"),
+                           ("comp", "f8"), ("count", "i8"), ("member", "i4"), ("pad_", "i4")])
+
+
+def round_to_storage(x: np.ndarray, dtype: int) -> np.ndarray:
+    """Round float32 values to the storage type (nearest, ties to even) and widen
+    them back to float64: F32 is the identity, BF16 keeps the upper 16 bits."""
+    x = np.asarray(x, dtype=np.float32)
+    if dtype == F32:
+        return x.astype(np.float64)
+    if dtype == F16:
+        return x.astype(np.float16).astype(np.float64)
+    bits = x.view(np.uint32).astype(np.uint64)
+    bits = (bits + 0x7FFF + ((bits >> 16) & 1)) & 0xFFFF0000        # nearest-even on the low half
+    return bits.astype(np.uint32).view(np.float32).astype(np.float64)
+
+
+def dvp_rows_listing(z: np.ndarray, ids: np.ndarray, rho: float, mask_value: float, *, dtype: int = F32,
+                     upstream: np.ndarray | None = None, threshold_in_storage_type: bool = True):
+    """The App. A listing taken literally (finite mask value kept in the partition
+    sum).  ``z`` holds the stored logits widened to float64.  The threshold is
+    max + log(rho), formed in float32 and rounded to the storage type when
+    ``threshold_in_storage_type`` is set, otherwise the exact double sum."""
+    lib = _load()
+    assert lib.dvp_oracle_sizeof_listing() == _LISTING_DTYPE.itemsize
+    lib.dvp_oracle_listing.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_double,
+                                       ctypes.c_double, ctypes.c_double, ctypes.c_void_p, ctypes.c_void_p]
+    lib.dvp_oracle_listing.restype = None
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    T, V = z.shape
+    log_rho = float(np.log(rho)) if rho > 0 else -np.inf
+    m = z.max(axis=1)
+    if threshold_in_storage_type:
+        with np.errstate(over="ignore"):
+            c = round_to_storage(np.array([log_rho], dtype=np.float32), dtype).astype(np.float32)[0]
+            thr = round_to_storage(m.astype(np.float32) + c, dtype)
+    else:
+        thr = m + log_rho
+    mv = float(round_to_storage(np.array([mask_value]), dtype)[0])
+    out = np.zeros(T, dtype=_LISTING_DTYPE)
+    grad = np.zeros((T, V)) if upstream is not None else None
+    ids = np.ascontiguousarray(ids, dtype=np.int64)
+    for t in range(T):
+        lib.dvp_oracle_listing(z.ctypes.data + t * V * 8, V, int(ids[t]), float(thr[t]), mv,
+                               float(upstream[t]) if upstream is not None else 0.0,
+                               out.ctypes.data + t * _LISTING_DTYPE.itemsize,
+                               grad.ctypes.data + t * V * 8 if grad is not None else None)
+    return out, grad, thr

@@ -261,6 +261,64 @@ int dvp_oracle_batch(const oracle_batch *b, int nthreads) {
 }
 
 /*
+ * The masking of the App. A listing, taken literally: pruned logits are not
+ * removed but replaced by a finite mask value (Sec. 5.5: "-50.0 in BF16"), which
+ * stays in the partition sum, and the threshold max + log(rho) is rounded to the
+ * logits' storage type before the strict comparison `logit < threshold`.
+ *   u_k = z_k if z_k >= thr else mask_value;  result = log_softmax(u)[a]
+ * The gradient flows only through kept positions (the mask value is a constant
+ * of `where`), the pruned ones get zero.  `thr` and `mask_value` arrive already
+ * rounded to the storage type by the caller.
+ */
+typedef struct {
+  double max, lse_full, lse_masked, logp_masked, comp; /* comp = 1 - softmax(u)_a */
+  int64_t count;                                        /* kept tokens            */
+  int32_t member, pad_;
+} oracle_listing;
+
+void dvp_oracle_listing(const double *z, int64_t V, int64_t a, double thr, double mask_value,
+                        double g, oracle_listing *out, double *grad) {
+  double m = -INFINITY;
+  for (int64_t k = 0; k < V; ++k)
+    if (z[k] > m) m = z[k];
+  const double top = m > mask_value ? m : mask_value;
+  nsum all = {0, 0}, masked = {0, 0}, masked_x = {0, 0};
+  int64_t n = 0;
+  for (int64_t k = 0; k < V; ++k) {
+    const int keep = !(z[k] < thr);
+    const double u = keep ? z[k] : mask_value;
+    nsum_add(&all, exp(z[k] - m));
+    nsum_add(&masked, exp(u - top));
+    if (k != a) nsum_add(&masked_x, exp(u - top));
+    n += keep;
+  }
+  const double s = nsum_value(&masked);
+  out->max = m;
+  out->lse_full = m + log(nsum_value(&all));
+  out->lse_masked = top + log(s);
+  out->count = n;
+  if (a >= 0 && a < V) {
+    const int keep_a = !(z[a] < thr);
+    out->member = keep_a;
+    out->logp_masked = (keep_a ? z[a] : mask_value) - out->lse_masked;
+    out->comp = nsum_value(&masked_x) / s;
+  } else {
+    out->member = 0;
+    out->logp_masked = NAN;
+    out->comp = NAN;
+  }
+  if (grad) {
+    for (int64_t k = 0; k < V; ++k) {
+      const int keep = !(z[k] < thr);
+      grad[k] = (a >= 0 && a < V && keep) ? -g * exp(z[k] - out->lse_masked) : 0.0;
+    }
+    if (a >= 0 && a < V && out->member) grad[a] = g * out->comp;
+  }
+}
+
+int dvp_oracle_sizeof_listing(void) { return (int)sizeof(oracle_listing); }
+
+/*
  * Sequence level (Sec. 4.4: Delta_y = sum_t Delta_{a_t}; Thm. 5.3: the ratio of a
  * trajectory is the product of its token ratios; App. A protocol 5: a token whose
  * importance weight pi^mp_train / pi^mp_infer falls below the veto threshold

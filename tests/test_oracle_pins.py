@@ -357,3 +357,39 @@ def test_sequence_level_ratio_is_the_product_of_token_ratios_and_veto_rule():
     res = oracle.dvp_sequences(np.array([0.0, math.log(1.01e-4), 0.1, math.log(0.99e-4), np.nan]),
                                np.array([0, 3, 5]), 1e-4)
     assert res.veto.tolist() == [0, 1] and res.n_valid.tolist() == [3, 1]
+
+
+@pytest.mark.parametrize("dt,code", [(torch.bfloat16, oracle.BF16), (torch.float32, oracle.F32)])
+def test_listing_variant_matches_torch_run_of_the_same_steps(dt, code):
+    """App. A taken literally: max, + log(rho) in the logits' dtype, strict <, where
+    with the finite mask value; then a float64 log-softmax and autograd."""
+    rng = np.random.default_rng(41)
+    T, V, rho, mv = 10, 400, 1e-2, -50.0
+    logits = torch.from_numpy((rng.normal(size=(T, V)) * 3).astype(np.float32)).to(dt)
+    with torch.no_grad():
+        threshold = logits.max(dim=-1, keepdim=True).values + math.log(rho)
+        pruned = logits < threshold
+    assert threshold.dtype == dt
+    z64 = logits.to(torch.float64).requires_grad_(True)
+    masked = torch.where(pruned, torch.tensor(mv, dtype=dt).to(torch.float64), z64)
+    ids = rng.integers(0, V, size=T)
+    ids[:3] = logits.float().numpy().argmax(1)[:3]
+    ids[3] = int(np.flatnonzero(pruned[3].numpy())[0])          # a pruned sampled token
+    g = torch.from_numpy(rng.normal(size=T))
+    logp = torch.log_softmax(masked, dim=-1)[torch.arange(T), torch.from_numpy(ids)]
+    (logp * g).sum().backward()
+    out, grad, thr = oracle.dvp_rows_listing(z64.detach().numpy(), ids, rho, mv, dtype=code, upstream=g.numpy())
+    np.testing.assert_array_equal(thr, threshold[:, 0].to(torch.float64).numpy())
+    np.testing.assert_array_equal(out["count"], (~pruned).sum(1).numpy())
+    np.testing.assert_allclose(out["logp_masked"], logp.detach().numpy(), atol=1e-12)
+    np.testing.assert_allclose(grad, z64.grad.numpy(), atol=1e-13)
+    assert out["member"][3] == 0 and np.isfinite(out["logp_masked"][3]) and np.abs(grad[3]).sum() > 0
+    # with rho small enough that nothing is pruned it is the plain log-softmax
+    out0, _, _ = oracle.dvp_rows_listing(z64.detach().numpy(), ids, 1e-30, mv, dtype=code)
+    ref = torch.log_softmax(z64.detach(), dim=-1)[torch.arange(T), torch.from_numpy(ids)].numpy()
+    np.testing.assert_allclose(out0["logp_masked"], ref, atol=1e-12)
+    # and it differs from the exact -inf semantics by the mass of the masked tokens
+    exact = oracle.dvp_rows_f64(z64.detach().numpy(), ids, rho)
+    kept = out["member"] == 1
+    extra = np.log1p((V - out["count"]) * np.exp(mv - exact.train.lse_safe))
+    np.testing.assert_allclose((exact.train.logp_mp - out["logp_masked"])[kept], extra[kept], atol=1e-9)
