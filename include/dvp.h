@@ -63,6 +63,21 @@ enum {
   DVP_FLAG_BAD_ID = 128  /* id >= V                                         */
 };
 
+/*
+ * bits of `mode` (dvp_forward_args, dvp_backward_args); 0 is the paper's definition.
+ *   DVP_MODE_FINITE_MASK  pruned logits are replaced by the finite `mask_value`
+ *       (rounded to the logits' type) and stay in the partition sum, as in the
+ *       listing of App. A and Sec. 5.5 ("-50.0 in BF16"): lse_safe becomes the
+ *       log-sum-exp of the masked row, logp_mp of a pruned sampled token is
+ *       mask_value - lse_safe (finite), log_ratio is always finite, and a pruned
+ *       sampled token still sends -g softmax(masked)_k to the kept positions.
+ *       Assumes max logit >= mask_value - 80.
+ *   DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE  the threshold is formed as an eager
+ *       tensor expression of the logits' type forms it: log(rho) rounded to that
+ *       type, added to the max in float32, the sum rounded to that type again.
+ */
+enum { DVP_MODE_FINITE_MASK = 1, DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE = 2 };
+
 enum { DVP_ENTRY_FORWARD = 0, DVP_ENTRY_BACKWARD = 1, DVP_ENTRY_FUSED_LMHEAD = 2 };
 
 /*
@@ -132,6 +147,8 @@ typedef struct {
   uint8_t *flags;
   void *stream;
   uint32_t launch_hint;
+  uint32_t mode;      /* DVP_MODE_* bits */
+  float mask_value;   /* used with DVP_MODE_FINITE_MASK */
   uint32_t reserved_;
 } dvp_forward_args;
 
@@ -165,6 +182,8 @@ typedef struct {
   void *grad_train;
   void *stream;
   uint32_t launch_hint;
+  uint32_t mode;      /* as in the dvp_forward call that saved the vectors */
+  float mask_value;
   uint32_t reserved_;
 } dvp_backward_args;
 

@@ -22,6 +22,7 @@ DVP_ID_I64, DVP_ID_I32 = 0, 1
 DVP_FLAG_IN_TRAIN, DVP_FLAG_IN_INFER, DVP_FLAG_NO_ID, DVP_FLAG_BAD_ID = 1, 2, 64, 128
 DVP_ENTRY_FORWARD, DVP_ENTRY_BACKWARD, DVP_ENTRY_FUSED_LMHEAD = 0, 1, 2
 DVP_STATIC_WORKSPACE_BYTES = 32 * 1024 * 1024
+DVP_MODE_FINITE_MASK, DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE = 1, 2
 
 EXPORTS = ("dvp_forward", "dvp_backward", "dvp_fused_lmhead_forward_backward",
            "dvp_fused_lmhead_forward_backward_static", "dvp_sequence_aggregate", "dvp_gemm_tn",
@@ -64,6 +65,8 @@ class ForwardArgs(ctypes.Structure):
         ("flags", ctypes.c_void_p),
         ("stream", ctypes.c_void_p),
         ("launch_hint", ctypes.c_uint32),
+        ("mode", ctypes.c_uint32),
+        ("mask_value", ctypes.c_float),
         ("reserved_", ctypes.c_uint32),
     ]
 
@@ -89,6 +92,8 @@ class BackwardArgs(ctypes.Structure):
         ("grad_train", ctypes.c_void_p),
         ("stream", ctypes.c_void_p),
         ("launch_hint", ctypes.c_uint32),
+        ("mode", ctypes.c_uint32),
+        ("mask_value", ctypes.c_float),
         ("reserved_", ctypes.c_uint32),
     ]
 
@@ -221,10 +226,15 @@ def _id_dtype(ids: torch.Tensor) -> int:
 def dvp_forward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, *,
                 infer_logits: torch.Tensor | None = None, upstream: torch.Tensor | None = None,
                 grad_train: torch.Tensor | None = None, grad_dtype: torch.dtype | None = None,
-                want_mask: bool = False, stream=None, launch_hint: int = 0, out=None):
+                want_mask: bool = False, stream=None, launch_hint: int = 0, out=None,
+                mask_value: float | None = None, threshold_in_logits_dtype: bool = False):
     """Pruned log-probabilities of the sampled tokens for the training and the
     inference logits (Def. 5.1, Def. 5.2), their log-ratio, and, when
     ``upstream`` is given, dLoss/dlogits (Prop. 5.4) in the same launch.
+
+    ``mask_value`` (finite) switches to the App. A listing's semantics: pruned
+    logits are replaced by it instead of by -inf; ``threshold_in_logits_dtype``
+    rounds the threshold the way an eager tensor expression would.
 
     Returns a namespace with ``train`` / ``infer`` (per-token tensors),
     ``log_ratio``, ``flags`` and ``grad_train``.  Pass the namespace of an
@@ -275,6 +285,9 @@ def dvp_forward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, *,
         a.ld_grad = grad_train.stride(0)
     a.stream = _stream(stream)
     a.launch_hint = launch_hint
+    a.mode = (DVP_MODE_FINITE_MASK if mask_value is not None else 0) | \
+        (DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE if threshold_in_logits_dtype else 0)
+    a.mask_value = float(mask_value) if mask_value is not None else 0.0
     st = lib.dvp_forward(ctypes.byref(a))
     if st != DVP_OK:
         raise DvpError(st, "dvp_forward")
@@ -284,7 +297,8 @@ def dvp_forward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, *,
 def dvp_backward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, upstream: torch.Tensor,
                  saved, *, grad_train: torch.Tensor | None = None,
                  grad_dtype: torch.dtype | None = None, use_comp: bool = True, stream=None,
-                 launch_hint: int = 0) -> torch.Tensor:
+                 launch_hint: int = 0, mask_value: float | None = None,
+                 threshold_in_logits_dtype: bool = False) -> torch.Tensor:
     """dLoss/dlogits from the vectors an earlier ``dvp_forward`` saved
     (``saved`` = its result namespace) and a per-token upstream gradient."""
     lib = load_library()
@@ -308,6 +322,9 @@ def dvp_backward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, upst
     a.grad_train = _ptr(grad_train)
     a.stream = _stream(stream)
     a.launch_hint = launch_hint
+    a.mode = (DVP_MODE_FINITE_MASK if mask_value is not None else 0) | \
+        (DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE if threshold_in_logits_dtype else 0)
+    a.mask_value = float(mask_value) if mask_value is not None else 0.0
     st = lib.dvp_backward(ctypes.byref(a))
     if st != DVP_OK:
         raise DvpError(st, "dvp_backward")

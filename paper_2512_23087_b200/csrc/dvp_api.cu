@@ -14,6 +14,11 @@ bool hint_ok(uint32_t hint) {
   return (stage == 0 || stage == 1 || stage == 2) && (cluster == 0 || cluster == 1 || cluster == 2 || cluster == 4);
 }
 
+bool mode_ok(uint32_t mode, float mask_value) {
+  if (mode & ~(uint32_t)(DVP_MODE_FINITE_MASK | DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE)) return false;
+  return !(mode & DVP_MODE_FINITE_MASK) || std::isfinite(mask_value);
+}
+
 bool side_empty(const dvp_side_out &o) {
   return !o.max && !o.lse && !o.lse_safe && !o.logp && !o.logp_mp && !o.comp_mp && !o.count &&
          !o.mask;
@@ -33,7 +38,7 @@ int dvp_forward(const dvp_forward_args *a) {
   if (a->T < 0 || a->T > 0x7fffffffLL || a->V < 1) return DVP_ERR_INVALID_ARG;
   if (a->V > 0x7fffff00LL) return DVP_ERR_UNSUPPORTED;
   if (!(a->rho >= 0.0 && a->rho <= 1.0)) return DVP_ERR_INVALID_ARG;
-  if (!hint_ok(a->launch_hint)) return DVP_ERR_INVALID_ARG;
+  if (!hint_ok(a->launch_hint) || !mode_ok(a->mode, a->mask_value)) return DVP_ERR_INVALID_ARG;
   if (a->T == 0) return DVP_OK;
   if (!a->train_logits || a->ld_train < a->V) return DVP_ERR_INVALID_ARG;
   if (a->infer_logits && a->ld_infer < a->V) return DVP_ERR_INVALID_ARG;
@@ -54,6 +59,8 @@ int dvp_forward(const dvp_forward_args *a) {
   p.ld_grad = a->ld_grad;
   p.log_rho = log_of_rho(a->rho);
   p.id_is_i32 = a->id_dtype == DVP_ID_I32;
+  p.mode = (int)a->mode;
+  p.mask_value = a->mask_value;
   p.out_t = a->train;
   p.out_i = a->infer;
   p.log_ratio = a->log_ratio;
@@ -70,7 +77,7 @@ int dvp_backward(const dvp_backward_args *a) {
   if (a->T < 0 || a->T > 0x7fffffffLL || a->V < 1) return DVP_ERR_INVALID_ARG;
   if (a->V > 0x7fffff00LL) return DVP_ERR_UNSUPPORTED;
   if (!(a->rho >= 0.0 && a->rho <= 1.0)) return DVP_ERR_INVALID_ARG;
-  if (!hint_ok(a->launch_hint)) return DVP_ERR_INVALID_ARG;
+  if (!hint_ok(a->launch_hint) || !mode_ok(a->mode, a->mask_value)) return DVP_ERR_INVALID_ARG;
   if (a->T == 0) return DVP_OK;
   if (!a->train_logits || !a->ids || !a->upstream || !a->max_t || !a->lse_safe_t || !a->flags ||
       !a->grad_train)
@@ -92,6 +99,8 @@ int dvp_backward(const dvp_backward_args *a) {
   p.ld_grad = a->ld_grad;
   p.log_rho = log_of_rho(a->rho);
   p.id_is_i32 = a->id_dtype == DVP_ID_I32;
+  p.mode = (int)a->mode;
+  p.mask_value = a->mask_value;
   const cudaError_t e = dvp::launch_backward_kernel(p, a->logits_dtype, a->grad_dtype,
                                                     a->launch_hint,
                                                     static_cast<cudaStream_t>(a->stream));

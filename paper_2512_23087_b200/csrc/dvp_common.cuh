@@ -293,6 +293,8 @@ struct RowParams {
   long long T, V, ld_train, ld_infer, ld_grad;
   double log_rho;  // ln(rho); -inf for rho = 0
   int id_is_i32;
+  int mode;          // DVP_MODE_* bits
+  float mask_value;  // finite mask value (DVP_MODE_FINITE_MASK)
   dvp_side_out out_t, out_i;
   float *log_ratio;
   uint8_t *flags;
@@ -310,29 +312,59 @@ __device__ __forceinline__ float threshold_f32(float m, double log_rho) {
   return __double2float_ru((double)m + log_rho);
 }
 
+// The threshold as an eager tensor expression of the logits' type forms it
+// (DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE), or the exact one.
+template <typename TIn>
+__device__ __forceinline__ float threshold_of(float m, double log_rho, int mode) {
+  if (mode & DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE) {
+    const float c = Storage<TIn>::widen(Storage<TIn>::narrow((float)log_rho));
+    return Storage<TIn>::widen(Storage<TIn>::narrow(m + c));
+  }
+  return threshold_f32(m, log_rho);
+}
+
 // Everything one side of one row reduces to.
 struct SideStats {
   float m;       // row max
   double lse;    // ln sum_k e^{z_k}
   float s_x;     // sum over the safe set of e^{z_k - m}, without the sampled token
   float e_a;     // e^{z_a - m} when a is in the safe set, else 0
+  float s_mask;  // mass of the masked tokens, (V - n) e^{mask_value - m}; 0 without a finite mask
+  float e_mask;  // e^{mask_value - m}; 0 without a finite mask
   float z_a;     // logit of the sampled token (0 when there is none)
-  float tau;     // threshold_f32(m, log_rho)
+  float tau;     // threshold
   int n;         // |V_S|
   int member;    // a in V_S
+  int live;      // the row has a gradient: a valid and (a in V_S or finite mask)
 };
+
+// Mass of the masked tokens once the count is known.
+__device__ __forceinline__ void set_mask_mass(SideStats &st, long long V, int mode, float mask_value_d,
+                                              bool has_a) {
+  st.e_mask = (mode & DVP_MODE_FINITE_MASK) ? ex2((mask_value_d - st.m) * kLog2e) : 0.f;
+  st.s_mask = (float)(V - st.n) * st.e_mask;
+  st.live = has_a && (st.member || (mode & DVP_MODE_FINITE_MASK));
+}
 
 // Writes the per-token outputs of one side; called by one thread.
 __device__ __forceinline__ float finish_side(const dvp_side_out &o, long long t, const SideStats &st,
                                              bool has_id, bool bad_id) {
-  const float s_safe = st.s_x + st.e_a;
-  const float log_ss = logf(s_safe);
+  const float s_tot = st.s_x + st.e_a + st.s_mask;
+  const float log_ss = logf(s_tot);
   const float nan = __int_as_float(0x7fc00000);
   float logp = nan, logp_mp = nan, comp = nan;
   if (has_id) {
     logp = (float)((double)st.z_a - st.lse);
-    logp_mp = st.member ? (st.z_a - st.m) - log_ss : kNegInf;
-    comp = st.member ? st.s_x / s_safe : 1.f;
+    if (st.member) {
+      logp_mp = (st.z_a - st.m) - log_ss;
+      comp = (st.s_x + st.s_mask) / s_tot;
+    } else if (st.e_mask > 0.f) {  // a masked token keeps the mask value's probability
+      logp_mp = logf(st.e_mask) - log_ss;
+      comp = (s_tot - st.e_mask) / s_tot;
+    } else {
+      logp_mp = kNegInf;
+      comp = 1.f;
+    }
   }
   if (bad_id) logp = logp_mp = comp = nan;
   if (o.max) o.max[t] = st.m;
@@ -361,6 +393,8 @@ struct BackwardParams {
   long long T, V, ld_train, ld_grad;
   double log_rho;
   int id_is_i32;
+  int mode;
+  float mask_value;
 };
 
 // Launchers (dvp_rows.cu).  `hint`: threads per block in the low 16 bits,

@@ -389,16 +389,16 @@ __device__ __forceinline__ SumCount row_sweep2(const TIn *row, int V, int a, flo
 // block sweeps the part [off, off + v_part) of it.
 template <typename TIn, int kStage, int kCluster>
 __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int off, int v_part, int a,
-                                               double log_rho, uint16_t *bound, float *scratch,
-                                               float *cl_slots, uint32_t *hot_smem, HotList &hot,
-                                               uint32_t *mask_row) {
+                                               double log_rho, int mode, float mask_value,
+                                               uint16_t *bound, float *scratch, float *cl_slots,
+                                               uint32_t *hot_smem, HotList &hot, uint32_t *mask_row) {
   const LogSum part = row_sweep1<TIn, kStage>(row + off, v_part, bound, scratch);
   const LogSum all = cluster_reduce_logsum<kCluster>(part, cl_slots);
 
   SideStats st;
   st.m = all.m;
   st.lse = lse_from_logsum(all);
-  st.tau = threshold_f32(all.m, log_rho);
+  st.tau = threshold_of<TIn>(all.m, log_rho, mode);
   const bool has_a = a >= 0 && a < V;
   st.z_a = has_a ? Storage<TIn>::widen(row[a]) : 0.f;
   st.member = has_a && st.z_a >= st.tau;
@@ -410,6 +410,7 @@ __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int off, i
   const SumCount tot = cluster_reduce_sumcount<kCluster>(sc, cl_slots + 4);
   st.s_x = tot.s;
   st.n = tot.n;
+  set_mask_mass(st, V, mode, Storage<TIn>::widen(Storage<TIn>::narrow(mask_value)), has_a);
 
   // ---- optional packed membership mask (diagnostic output, plain loads)
   if (mask_row && off == 0) {
@@ -438,12 +439,13 @@ __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int
   const int per_step = kStage * (int)blockDim.x;
   const int n_slots = ((n_gran + per_step - 1) / per_step) * kStage;
   const int tid = threadIdx.x;
-  const float s_safe = st.s_x + st.e_a;
-  // a pruned or missing sampled token has weight zero: the row is all zeros
-  const bool live = st.member;
-  const float coef = live ? -g / s_safe : 0.f;
-  const float g_a = live ? g * (st.s_x / s_safe) : 0.f;
-  const int a_live = live ? a : -1;
+  const float s_tot = st.s_x + st.e_a + st.s_mask;
+  // a missing sampled token, or a pruned one under the -inf semantics, has weight zero:
+  // the row is all zeros
+  const bool live = st.live;
+  const float coef = live ? -g / s_tot : 0.f;
+  const float g_a = st.member ? g * ((st.s_x + st.s_mask) / s_tot) : 0.f;
+  const int a_live = (live && st.member) ? a : -1;
   const bool listed = live && hot.fits();
   const float tau = live ? st.tau : -kNegInf;  // +inf: nothing passes
 
@@ -514,8 +516,9 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
   const TIn *trow = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
   uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * ((p.V + 31) / 32) : nullptr;
   HotList hot;
-  const SideStats st = row_stats<TIn, kStage, kCluster>(trow, V, off, v_part, a, p.log_rho, bound,
-                                                        scratch, cl_slots, hot_smem, hot, mask_t);
+  const SideStats st =
+      row_stats<TIn, kStage, kCluster>(trow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value, bound,
+                                       scratch, cl_slots, hot_smem, hot, mask_t);
 
   if (p.grad) {
     const float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
@@ -530,8 +533,8 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
     const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
     uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
     HotList hot_i;
-    si = row_stats<TIn, kStage, kCluster>(irow, V, off, v_part, a, p.log_rho, bound, scratch,
-                                          cl_slots + 8, hot_smem, hot_i, mask_i);
+    si = row_stats<TIn, kStage, kCluster>(irow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value,
+                                          bound, scratch, cl_slots + 8, hot_smem, hot_i, mask_i);
   }
 
   if (threadIdx.x == 0 && rank == 0) {
@@ -542,8 +545,9 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
       const float li = finish_side(p.out_i, t, si, has_id, bad_id);
       if (si.member) flags |= DVP_FLAG_IN_INFER;
       if (p.log_ratio)
-        p.log_ratio[t] = (has_id && !bad_id) ? log_ratio_of(st.member, si.member, lt, li)
-                                             : __int_as_float(0x7fc00000);
+        p.log_ratio[t] = !(has_id && !bad_id)              ? __int_as_float(0x7fc00000)
+                         : (p.mode & DVP_MODE_FINITE_MASK) ? lt - li
+                                                           : log_ratio_of(st.member, si.member, lt, li);
     }
     if (p.flags) p.flags[t] = flags;
   }
@@ -557,8 +561,8 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
 
 template <typename TIn>
 __device__ __forceinline__ SideStats row_stats_scalar(const TIn *row, long long V, long long a,
-                                                      double log_rho, float *scratch,
-                                                      uint32_t *mask_row) {
+                                                      double log_rho, int mode, float mask_value,
+                                                      float *scratch, uint32_t *mask_row) {
   float m = kNegInf;
   for (long long k = threadIdx.x; k < V; k += blockDim.x) m = fmaxf(m, Storage<TIn>::widen(row[k]));
   MaxSum acc = {m, 0.f};
@@ -569,7 +573,7 @@ __device__ __forceinline__ SideStats row_stats_scalar(const TIn *row, long long 
   SideStats st;
   st.m = all.m;
   st.lse = (double)all.m + (double)logf(all.s);
-  st.tau = threshold_f32(all.m, log_rho);
+  st.tau = threshold_of<TIn>(all.m, log_rho, mode);
   const bool has_a = a >= 0 && a < V;
   st.z_a = has_a ? Storage<TIn>::widen(row[a]) : 0.f;
   st.member = has_a && st.z_a >= st.tau;
@@ -585,6 +589,7 @@ __device__ __forceinline__ SideStats row_stats_scalar(const TIn *row, long long 
   const SumCount tot = block_reduce_sumcount(sc, scratch);
   st.s_x = tot.s;
   st.n = tot.n;
+  set_mask_mass(st, V, mode, Storage<TIn>::widen(Storage<TIn>::narrow(mask_value)), has_a);
   if (mask_row) {
     const long long n_words = (V + 31) / 32;
     for (long long w = threadIdx.x; w < n_words; w += blockDim.x) {
@@ -609,19 +614,20 @@ __global__ void dvp_row_kernel_scalar(const RowParams p) {
 
   const TIn *trow = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
   uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * ((p.V + 31) / 32) : nullptr;
-  const SideStats st = row_stats_scalar<TIn>(trow, p.V, a, p.log_rho, scratch, mask_t);
+  const SideStats st =
+      row_stats_scalar<TIn>(trow, p.V, a, p.log_rho, p.mode, p.mask_value, scratch, mask_t);
 
   if (p.grad) {
     TGrad *grow = reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad;
     const float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
-    const float s_safe = st.s_x + st.e_a;
-    const bool live = st.member;
-    const float coef = live ? -g / s_safe : 0.f;
-    const float g_a = live ? g * (st.s_x / s_safe) : 0.f;
+    const float s_tot = st.s_x + st.e_a + st.s_mask;
+    const bool live = st.live;
+    const float coef = live ? -g / s_tot : 0.f;
+    const float g_a = st.member ? g * ((st.s_x + st.s_mask) / s_tot) : 0.f;
     for (long long k = threadIdx.x; k < p.V; k += blockDim.x) {
       const float z = Storage<TIn>::widen(trow[k]);
       float out = (live && z >= st.tau) ? coef * ex2((z - st.m) * kLog2e) : 0.f;
-      if (live && k == a) out = g_a;
+      if (live && st.member && k == a) out = g_a;
       grow[k] = Storage<TGrad>::narrow(out);
     }
   }
@@ -630,7 +636,7 @@ __global__ void dvp_row_kernel_scalar(const RowParams p) {
   if (p.infer) {
     const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
     uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
-    si = row_stats_scalar<TIn>(irow, p.V, a, p.log_rho, scratch, mask_i);
+    si = row_stats_scalar<TIn>(irow, p.V, a, p.log_rho, p.mode, p.mask_value, scratch, mask_i);
   }
 
   if (threadIdx.x == 0) {
@@ -641,8 +647,9 @@ __global__ void dvp_row_kernel_scalar(const RowParams p) {
       const float li = finish_side(p.out_i, t, si, has_id, bad_id);
       if (si.member) flags |= DVP_FLAG_IN_INFER;
       if (p.log_ratio)
-        p.log_ratio[t] = (has_id && !bad_id) ? log_ratio_of(st.member, si.member, lt, li)
-                                             : __int_as_float(0x7fc00000);
+        p.log_ratio[t] = !(has_id && !bad_id)              ? __int_as_float(0x7fc00000)
+                         : (p.mode & DVP_MODE_FINITE_MASK) ? lt - li
+                                                           : log_ratio_of(st.member, si.member, lt, li);
     }
     if (p.flags) p.flags[t] = flags;
   }
@@ -656,14 +663,16 @@ __global__ void dvp_backward_kernel(const BackwardParams p) {
   const TIn *row = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
   TGrad *grow = reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad;
   const long long id = load_id(p.ids, p.id_is_i32, t);
-  const bool live = (p.flags[t] & DVP_FLAG_IN_TRAIN) && id >= 0 && id < p.V;
-  const long long a = live ? id : -1;
+  const bool member = (p.flags[t] & DVP_FLAG_IN_TRAIN) && id >= 0 && id < p.V;
+  // with a finite mask value a pruned sampled token still has a gradient on the kept positions
+  const bool live = member || ((p.mode & DVP_MODE_FINITE_MASK) && id >= 0 && id < p.V);
+  const long long a = member ? id : -1;
   const float g = p.upstream[t], m = p.max_t[t];
-  const float tau = live ? threshold_f32(m, p.log_rho) : -kNegInf;
+  const float tau = live ? threshold_of<TIn>(m, p.log_rho, p.mode) : -kNegInf;
   // e^{z - lse_safe} = e^{z - m} e^{m - lse_safe}; the second factor is 1 / s_safe
   const float coef = live ? -g * ex2((m - p.lse_safe_t[t]) * kLog2e) : 0.f;
   float g_a = 0.f;
-  if (live) {
+  if (member) {
     const float comp = p.comp_mp_t ? p.comp_mp_t[t]
                                    : -expm1f(Storage<TIn>::widen(row[a]) - p.lse_safe_t[t]);
     g_a = g * comp;
