@@ -369,3 +369,21 @@ def dvp_rows_listing(z: np.ndarray, ids: np.ndarray, rho: float, mask_value: flo
                                out.ctypes.data + t * _LISTING_DTYPE.itemsize,
                                grad.ctypes.data + t * V * 8 if grad is not None else None)
     return out, grad, thr
+
+
+def dvp_monitor(z: np.ndarray, zi: np.ndarray) -> np.ndarray:
+    """Per-token KL(infer || train), KL(train || infer), H(train), H(infer) in nats over
+    the full vocabulary; ``z`` and ``zi`` are the stored logits widened to float64.
+    Returns a [T, 4] array."""
+    lib = _load()
+    lib.dvp_oracle_monitor.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]
+    lib.dvp_oracle_monitor.restype = None
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    zi = np.ascontiguousarray(zi, dtype=np.float64)
+    assert z.shape == zi.shape and z.ndim == 2
+    T, V = z.shape
+    out = np.zeros((T, 4))
+    for t in range(T):
+        lib.dvp_oracle_monitor(z.ctypes.data + t * V * 8, zi.ctypes.data + t * V * 8, V,
+                               out.ctypes.data + t * 32)
+    return out

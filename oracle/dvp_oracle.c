@@ -316,6 +316,41 @@ void dvp_oracle_listing(const double *z, int64_t V, int64_t a, double thr, doubl
   }
 }
 
+/*
+ * Monitoring quantities of one token: the Kullback-Leibler divergences between
+ * the full-vocabulary inference and training policies (the stability metric of
+ * Sec. 6) and their entropies (the quantity Sec. 7 proposes to adapt rho to).
+ *   KL(p || q) = sum_k p_k (ln p_k - ln q_k),   H(p) = - sum_k p_k ln p_k,
+ * with p = softmax(z), written out term by term.
+ * out: kl_infer_train, kl_train_infer, entropy_train, entropy_infer.
+ */
+void dvp_oracle_monitor(const double *z, const double *zi, int64_t V, double *out) {
+  double m = -INFINITY, mi = -INFINITY;
+  for (int64_t k = 0; k < V; ++k) {
+    if (z[k] > m) m = z[k];
+    if (zi[k] > mi) mi = zi[k];
+  }
+  nsum s = {0, 0}, si = {0, 0};
+  for (int64_t k = 0; k < V; ++k) {
+    nsum_add(&s, exp(z[k] - m));
+    nsum_add(&si, exp(zi[k] - mi));
+  }
+  const double lse = m + log(nsum_value(&s)), lsei = mi + log(nsum_value(&si));
+  nsum kl_it = {0, 0}, kl_ti = {0, 0}, h_t = {0, 0}, h_i = {0, 0};
+  for (int64_t k = 0; k < V; ++k) {
+    const double lp = z[k] - lse, lq = zi[k] - lsei; /* ln pi_train(k), ln pi_infer(k) */
+    const double p = exp(lp), q = exp(lq);
+    if (q > 0) nsum_add(&kl_it, q * (lq - lp));
+    if (p > 0) nsum_add(&kl_ti, p * (lp - lq));
+    if (p > 0) nsum_add(&h_t, -p * lp);
+    if (q > 0) nsum_add(&h_i, -q * lq);
+  }
+  out[0] = nsum_value(&kl_it);
+  out[1] = nsum_value(&kl_ti);
+  out[2] = nsum_value(&h_t);
+  out[3] = nsum_value(&h_i);
+}
+
 int dvp_oracle_sizeof_listing(void) { return (int)sizeof(oracle_listing); }
 
 /*

@@ -393,3 +393,33 @@ def test_listing_variant_matches_torch_run_of_the_same_steps(dt, code):
     kept = out["member"] == 1
     extra = np.log1p((V - out["count"]) * np.exp(mv - exact.train.lse_safe))
     np.testing.assert_allclose((exact.train.logp_mp - out["logp_masked"])[kept], extra[kept], atol=1e-9)
+
+
+def test_monitoring_quantities_against_library_routines_and_invariants():
+    """Sec. 6 monitors the KL divergence between the inference and training
+    policies; the oracle's values are pinned to torch's kl_div and Categorical
+    entropy, to KL >= 0 with equality for equal rows, to shift invariance, and to
+    the second-order value Var_pi(eps) / 2 for a small perturbation eps."""
+    rng = np.random.default_rng(43)
+    T, V = 9, 700
+    z = _rows(rng, T, V, scale=3.0)
+    zi = z + rng.normal(size=z.shape) * 0.3
+    got = oracle.dvp_monitor(z, zi)
+    lt, li = torch.log_softmax(torch.from_numpy(z), -1), torch.log_softmax(torch.from_numpy(zi), -1)
+    kl_it = torch.nn.functional.kl_div(lt, li, log_target=True, reduction="none").sum(-1).numpy()
+    kl_ti = torch.nn.functional.kl_div(li, lt, log_target=True, reduction="none").sum(-1).numpy()
+    np.testing.assert_allclose(got[:, 0], kl_it, atol=1e-12)
+    np.testing.assert_allclose(got[:, 1], kl_ti, atol=1e-12)
+    np.testing.assert_allclose(got[:, 2], torch.distributions.Categorical(logits=torch.from_numpy(z)).entropy().numpy(), atol=1e-12)
+    np.testing.assert_allclose(got[:, 3], torch.distributions.Categorical(logits=torch.from_numpy(zi)).entropy().numpy(), atol=1e-12)
+    assert (got[:, :2] > 0).all() and (got[:, 2:] <= math.log(V) + 1e-12).all()
+    same = oracle.dvp_monitor(z, z + 7.5)                      # softmax ignores a shift of the row
+    np.testing.assert_allclose(same[:, :2], 0.0, atol=1e-12)
+    np.testing.assert_allclose(same[:, 2], same[:, 3], atol=1e-12)
+    eps = rng.normal(size=z.shape) * 1e-3
+    small = oracle.dvp_monitor(z, z + eps)
+    pi = torch.softmax(torch.from_numpy(z), -1).numpy()
+    var = (pi * eps ** 2).sum(1) - (pi * eps).sum(1) ** 2
+    np.testing.assert_allclose(small[:, 0], var / 2, rtol=5e-3)
+    flat = oracle.dvp_monitor(np.zeros((1, 64)), np.zeros((1, 64)))
+    assert flat[0, 2] == pytest.approx(math.log(64), abs=1e-14)
