@@ -288,6 +288,32 @@ typedef struct {
 int dvp_sequence_aggregate(const dvp_sequence_args *args);
 
 /*
+ * dvp_monitor -- per-token monitoring quantities over the full vocabulary: the
+ * Kullback-Leibler divergences between the inference and the training policy
+ * (the training-stability metric of Sec. 6) and the entropy of each (the
+ * quantity Sec. 7 proposes to adapt rho to), in nats:
+ *   KL(p || q) = sum_k p_k (ln p_k - ln q_k),  H(p) = -sum_k p_k ln p_k,
+ *   pi_train = softmax(train_logits[t]), pi_infer = softmax(infer_logits[t]).
+ * Both matrices are read once.  Each output is a device [T] float32 array and
+ * may be NULL.  Rows that start on 32-byte boundaries take the vectorised
+ * kernel, other layouts a scalar one.  Errors as in dvp_forward.
+ */
+typedef struct {
+  uint32_t struct_size;
+  int32_t logits_dtype;
+  int64_t T, V, ld_train, ld_infer;
+  const void *train_logits;
+  const void *infer_logits;
+  float *kl_infer_train; /* KL(pi_infer || pi_train) */
+  float *kl_train_infer; /* KL(pi_train || pi_infer) */
+  float *entropy_train;
+  float *entropy_infer;
+  void *stream;
+} dvp_monitor_args;
+
+int dvp_monitor(const dvp_monitor_args *args);
+
+/*
  * dvp_fused_lmhead_forward_backward_static -- the fused entry point for callers
  * that cannot obtain device memory of their own.  (The paper has no counterpart;
  * this is a packaging variant of the entry point above.)

@@ -25,7 +25,7 @@ DVP_STATIC_WORKSPACE_BYTES = 32 * 1024 * 1024
 DVP_MODE_FINITE_MASK, DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE = 1, 2
 
 EXPORTS = ("dvp_forward", "dvp_backward", "dvp_fused_lmhead_forward_backward",
-           "dvp_fused_lmhead_forward_backward_static", "dvp_sequence_aggregate", "dvp_gemm_tn",
+           "dvp_fused_lmhead_forward_backward_static", "dvp_sequence_aggregate", "dvp_monitor", "dvp_gemm_tn",
            "dvp_workspace_bytes", "dvp_status_string", "dvp_version")
 
 _DTYPES = {torch.float32: DVP_F32, torch.bfloat16: DVP_BF16, torch.float16: DVP_F16}
@@ -148,6 +148,24 @@ class SequenceArgs(ctypes.Structure):
     ]
 
 
+class MonitorArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("logits_dtype", ctypes.c_int32),
+        ("T", ctypes.c_int64),
+        ("V", ctypes.c_int64),
+        ("ld_train", ctypes.c_int64),
+        ("ld_infer", ctypes.c_int64),
+        ("train_logits", ctypes.c_void_p),
+        ("infer_logits", ctypes.c_void_p),
+        ("kl_infer_train", ctypes.c_void_p),
+        ("kl_train_infer", ctypes.c_void_p),
+        ("entropy_train", ctypes.c_void_p),
+        ("entropy_infer", ctypes.c_void_p),
+        ("stream", ctypes.c_void_p),
+    ]
+
+
 _lib = None
 
 
@@ -170,6 +188,8 @@ def load_library() -> ctypes.CDLL:
         lib.dvp_fused_lmhead_forward_backward_static.restype = ctypes.c_int
         lib.dvp_sequence_aggregate.argtypes = [ctypes.POINTER(SequenceArgs)]
         lib.dvp_sequence_aggregate.restype = ctypes.c_int
+        lib.dvp_monitor.argtypes = [ctypes.POINTER(MonitorArgs)]
+        lib.dvp_monitor.restype = ctypes.c_int
         lib.dvp_gemm_tn.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64,
                                     ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int64, ctypes.c_int32, ctypes.c_float, ctypes.c_int32,
@@ -492,4 +512,31 @@ def dvp_sequence_aggregate(log_ratio: torch.Tensor, seq_offsets: torch.Tensor,
     st = lib.dvp_sequence_aggregate(ctypes.byref(a))
     if st != DVP_OK:
         raise DvpError(st, "dvp_sequence_aggregate")
+    return res
+
+
+def dvp_monitor(train_logits: torch.Tensor, infer_logits: torch.Tensor, stream=None):
+    """Per-token KL(infer || train), KL(train || infer) and the two entropies over
+    the full vocabulary (Sec. 6's stability metric), in nats."""
+    lib = load_library()
+    _check_matrix("train_logits", train_logits)
+    _check_matrix("infer_logits", infer_logits)
+    if infer_logits.dtype != train_logits.dtype or infer_logits.shape != train_logits.shape:
+        raise ValueError("infer_logits must match train_logits in dtype and shape")
+    T, V = train_logits.shape
+    dev = train_logits.device
+    res = SimpleNamespace(**{n: torch.empty(T, dtype=torch.float32, device=dev)
+                             for n in ("kl_infer_train", "kl_train_infer", "entropy_train", "entropy_infer")})
+    a = MonitorArgs()
+    a.struct_size = ctypes.sizeof(MonitorArgs)
+    a.logits_dtype = _DTYPES[train_logits.dtype]
+    a.T, a.V = T, V
+    a.ld_train, a.ld_infer = train_logits.stride(0), infer_logits.stride(0)
+    a.train_logits, a.infer_logits = _ptr(train_logits), _ptr(infer_logits)
+    a.kl_infer_train, a.kl_train_infer = _ptr(res.kl_infer_train), _ptr(res.kl_train_infer)
+    a.entropy_train, a.entropy_infer = _ptr(res.entropy_train), _ptr(res.entropy_infer)
+    a.stream = _stream(stream)
+    st = lib.dvp_monitor(ctypes.byref(a))
+    if st != DVP_OK:
+        raise DvpError(st, "dvp_monitor")
     return res

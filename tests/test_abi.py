@@ -38,7 +38,7 @@ def test_struct_layout_matches_the_header(tmp_path):
     from paper_2512_23087_b200 import binding
     structs = {"dvp_forward_args": binding.ForwardArgs, "dvp_backward_args": binding.BackwardArgs,
                "dvp_fused_args": binding.FusedArgs, "dvp_side_out": binding.SideOut,
-               "dvp_sequence_args": binding.SequenceArgs}
+               "dvp_sequence_args": binding.SequenceArgs, "dvp_monitor_args": binding.MonitorArgs}
     lines = []
     for cname, cls in structs.items():
         lines.append(f'printf("{cname} %zu\\n", sizeof({cname}));')
