@@ -115,9 +115,10 @@ typedef struct {
  *                 after Thm. 5.3), +inf when a is in V_S but outside V'_S
  *   flags         device [T] bytes, DVP_FLAG_* bits
  *   launch_hint   0 = library default; otherwise threads per block (a multiple
- *                 of 32, at most 512) in the low 16 bits and 32-byte loads per
- *                 thread and pipeline stage (1, 2 or 4) in the next 8 bits;
- *                 tuning only, the safe set and counts do not depend on it
+ *                 of 32, at most 512) in the low 16 bits, 0 or 2 in the next 8
+ *                 bits, and the number of blocks that share one row (0, 1, 2 or
+ *                 4; a thread-block cluster) in the top 8 bits; tuning only, the
+ *                 safe set and counts do not depend on it
  *
  * Rows whose start is 32-byte aligned in all three matrices take the
  * vectorised kernels; any other layout takes a scalar kernel, same results.

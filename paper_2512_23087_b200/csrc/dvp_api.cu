@@ -11,7 +11,7 @@ bool hint_ok(uint32_t hint) {
   const uint32_t threads = hint & 0xffff, stage = (hint >> 16) & 0xff;
   if (threads != 0 && (threads % 32 != 0 || threads > 512)) return false;
   const uint32_t cluster = (hint >> 24) & 0xff;
-  return (stage == 0 || stage == 1 || stage == 2) && (cluster == 0 || cluster == 1 || cluster == 2 || cluster == 4);
+  return (stage == 0 || stage == 2) && (cluster == 0 || cluster == 1 || cluster == 2 || cluster == 4);
 }
 
 bool mode_ok(uint32_t mode, float mask_value) {

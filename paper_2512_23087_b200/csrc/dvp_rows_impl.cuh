@@ -89,6 +89,18 @@ __device__ __forceinline__ uint16_t bf16_bits_round_up(float v) {
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
   return __uint_as_float((uint32_t)b << 16);
 }
+// Largest bfloat16 that is <= v, as a float: comparing the stored upper bounds with
+// it flags a superset of the granules whose bound reaches v.
+__device__ __forceinline__ float bf16_round_down(float v) {
+  const uint32_t b = __float_as_uint(v);
+  return __uint_as_float(((b & 0x80000000u) ? b + 0xffffu : b) & 0xffff0000u);
+}
+// The bounds of one thread's kStage granules of a step sit side by side, so that a
+// step's pair is one 32-bit word: slot i = step * kStage + u of thread tid.
+template <int kStage>
+__device__ __forceinline__ int bound_index(int slot, int tid) {
+  return ((slot / kStage) * (int)blockDim.x + tid) * kStage + (slot % kStage);
+}
 
 template <typename TGrad, int kElems>
 __device__ __forceinline__ void store_granule(TGrad *dst, const float *out) {
@@ -147,20 +159,45 @@ struct HotList {
   __device__ __forceinline__ bool fits() const { return count <= kHotCap; }
 };
 
-__device__ __forceinline__ HotList build_hot_list(const uint16_t *bound, int n_slots, float tau,
+// tau_b: the threshold rounded down to bfloat16.  Each thread first gathers the
+// flags of its own slots into a register (16 steps at a time: one packed compare per
+// step), then a warp prefix sum hands out list positions: the cost of the scan does
+// not depend on how many granules are hot, and the order of the list is fixed.
+template <int kStage>
+__device__ __forceinline__ HotList build_hot_list(const uint16_t *bound, int n_steps, float tau_b,
                                                   uint32_t *hot_smem) {
-  const int lane = threadIdx.x & 31;
+  static_assert(kStage == 2, "the packed scan reads the two bounds of a step as one word");
+  const int lane = threadIdx.x & 31, tid = threadIdx.x;
   HotList h;
-  h.slots = hot_smem + (threadIdx.x >> 5) * kHotCap;
+  h.slots = hot_smem + (tid >> 5) * kHotCap;
   h.count = 0;
-  for (int i = 0; i < n_slots; ++i) {
-    const bool f = bf16_bits_to_float(bound[i * blockDim.x + threadIdx.x]) >= tau;
-    const unsigned b = __ballot_sync(0xffffffffu, f);
-    if (f) {
-      const int pos = h.count + __popc(b & ((1u << lane) - 1u));
-      if (pos < kHotCap) h.slots[pos] = (uint32_t)(i * 32 + lane);
+  const uint32_t *words = reinterpret_cast<const uint32_t *>(bound);
+  const __nv_bfloat16 tb = __float2bfloat16_rz(tau_b);  // exact: tau_b is a bfloat16 value
+  const __nv_bfloat162 tau2 = __halves2bfloat162(tb, tb);
+  for (int step0 = 0; step0 < n_steps; step0 += 16) {
+    uint32_t acc = 0;  // bit s: first granule of step step0 + s, bit 16 + s: second granule
+    const int n = min(16, n_steps - step0);
+    for (int s = 0; s < n; ++s) {
+      const uint32_t w = words[(step0 + s) * blockDim.x + tid];
+      const uint32_t m = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&w), tau2);
+      acc |= (m & 0x00010001u) << s;
     }
-    h.count += __popc(b);
+    const int cnt = __popc(acc);
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    int pos = h.count + incl - cnt;
+    while (acc) {
+      const int b = __ffs(acc) - 1;
+      acc &= acc - 1;
+      const int slot = (step0 + (b & 15)) * 2 + (b >> 4);
+      if (pos < kHotCap) h.slots[pos] = (uint32_t)(slot * 32 + lane);
+      ++pos;
+    }
+    h.count += __shfl_sync(0xffffffffu, incl, 31);
   }
   __syncwarp();
   return h;
@@ -177,7 +214,7 @@ __device__ __forceinline__ void granule_masked_sum(const Granule<TIn> &gr, int g
   const int ja = a - g * kElems;  // in [0, kElems) only inside the owner granule
 #pragma unroll
   for (int j = 0; j < kElems; ++j) {
-    if (x[j] >= tau) {
+    if (x[j] >= tau && x[j] > kNegInf) {  // the fill of a ragged last granule is never a token
       ++sc.n;
       if (j != ja) sc.s += ex2((x[j] - m) * kLog2e);
     }
@@ -234,7 +271,7 @@ __device__ __forceinline__ void absorb_stage(const Stage<TIn, kStage> &st, int s
 #pragma unroll
   for (int u = 0; u < kStage; ++u) {
     const float gm = st.g[u].max();
-    bound[(step * kStage + u) * blockDim.x + threadIdx.x] = bf16_bits_round_up(gm);
+    bound[bound_index<kStage>(step * kStage + u, threadIdx.x)] = bf16_bits_round_up(gm);
     cm = fmaxf(cm, gm);
   }
   if (cm > kNegInf) {
@@ -357,7 +394,8 @@ __device__ __forceinline__ SumCount row_sweep2(const TIn *row, int V, int a, flo
   const int n_slots = ((n_gran + per_step - 1) / per_step) * kStage;  // granules per thread
   const int tid = threadIdx.x;
   SumCount sc = {0.f, 0};
-  hot = build_hot_list(bound, n_slots, tau, hot_smem);
+  const float tau_b = bf16_round_down(tau);
+  hot = build_hot_list<kStage>(bound, n_slots / kStage, tau_b, hot_smem);
   if (hot.fits()) {
     const int wbase = tid & ~31, lane = tid & 31;
     for (int q = lane; q < hot.count; q += 64) {
@@ -374,7 +412,7 @@ __device__ __forceinline__ SumCount row_sweep2(const TIn *row, int V, int a, flo
     }
   } else {
     for (int i = 0; i < n_slots; ++i) {
-      if (bf16_bits_to_float(bound[i * blockDim.x + tid]) >= tau) {
+      if (bf16_bits_to_float(bound[bound_index<kStage>(i, tid)]) >= tau_b) {
         const int g = i * (int)blockDim.x + tid;
         Granule<TIn> gr;
         gr.load_any(row, V, n_full, g);
@@ -448,11 +486,12 @@ __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int
   const int a_live = (live && st.member) ? a : -1;
   const bool listed = live && hot.fits();
   const float tau = live ? st.tau : -kNegInf;  // +inf: nothing passes
+  const float tau_b = live ? bf16_round_down(st.tau) : -kNegInf;
 
   for (int i = 0; i < n_slots; ++i) {
     const int gi = i * (int)blockDim.x + tid;
     if (gi >= n_gran) break;
-    if (bf16_bits_to_float(bound[i * blockDim.x + tid]) >= tau) {
+    if (bf16_bits_to_float(bound[bound_index<kStage>(i, tid)]) >= tau_b) {
       if (!listed) {
         Granule<TIn> gr;
         gr.load_any(row, V, n_full, gi);
@@ -748,7 +787,7 @@ static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s
   // measured on B200: 4-byte logits run best with 2 x 512 threads per SM, 2-byte
   // logits (twice the exponentials per byte) with 4 x 256
   if (threads == 0) threads = sizeof(TIn) == 4 ? 512 : 256;
-  if (stage == 0) stage = 2;
+  stage = 2;  // two granules per thread and pipeline stage
   const bool vec_ok = aligned32(p.train, p.ld_train, sizeof(TIn)) &&
                       aligned32(p.infer, p.ld_infer, sizeof(TIn)) &&
                       aligned32(p.grad, p.ld_grad, sizeof(TGrad));
@@ -766,11 +805,7 @@ static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s
       return launch_rows_vec<TIn, TGrad, 2, 256, 4, 4>(p, threads, smem, s);
     if (cluster == 2 && threads <= 256 && stage == 2)
       return launch_rows_vec<TIn, TGrad, 2, 256, 4, 2>(p, threads, smem, s);
-    if (threads > 256) {
-      if (stage == 1) return launch_rows_vec<TIn, TGrad, 1, 512, 2, 1>(p, threads, smem, s);
-      return launch_rows_vec<TIn, TGrad, 2, 512, 2, 1>(p, threads, smem, s);
-    }
-    if (stage == 1) return launch_rows_vec<TIn, TGrad, 1, 256, 4, 1>(p, threads, smem, s);
+    if (threads > 256) return launch_rows_vec<TIn, TGrad, 2, 512, 2, 1>(p, threads, smem, s);
     return launch_rows_vec<TIn, TGrad, 2, 256, 4, 1>(p, threads, smem, s);
   }
   dvp_row_kernel_scalar<TIn, TGrad><<<(unsigned)p.T, 512, 0, s>>>(p);
