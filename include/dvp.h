@@ -375,6 +375,21 @@ int dvp_gemm_tn(const void *a, int64_t lda, const void *b, int64_t ldb, float *c
                 int32_t *status, void *stream);
 
 /*
+ * dvp_row_wait_status -- the row kernel that keeps rows resident in shared
+ * memory (launch_hint stage byte 0x11 / 0x12, and the default for row shapes it
+ * serves) waits on hardware barriers for its bulk copies and for the other
+ * blocks of its cluster.  Every such wait is bounded; one that runs out ends the
+ * launch early (outputs of that launch are then undefined) and ORs a code into a
+ * per-device status word: 1 a copy did not land, 2 a ring slot was not handed
+ * back, 4 a block of the cluster did not report.  This call waits for all work
+ * on the current device (it synchronises), copies the word to *status_out (a
+ * host pointer) and clears it.  The paper has no counterpart.  0 means that no
+ * wait has run out since the last call.  Errors: DVP_ERR_INVALID_ARG (NULL),
+ * DVP_ERR_CUDA.
+ */
+int dvp_row_wait_status(uint32_t *status_out);
+
+/*
  * Bytes of device workspace the entry point needs for `args` (a pointer to
  * that entry point's args struct; only sizes and dtypes are read).  Returns 0
  * for entry points that need none and for invalid arguments.

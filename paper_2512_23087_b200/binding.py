@@ -26,7 +26,7 @@ DVP_MODE_FINITE_MASK, DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE = 1, 2
 
 EXPORTS = ("dvp_forward", "dvp_backward", "dvp_fused_lmhead_forward_backward",
            "dvp_fused_lmhead_forward_backward_static", "dvp_sequence_aggregate", "dvp_monitor", "dvp_gemm_tn",
-           "dvp_workspace_bytes", "dvp_status_string", "dvp_version")
+           "dvp_workspace_bytes", "dvp_status_string", "dvp_version", "dvp_row_wait_status")
 
 _DTYPES = {torch.float32: DVP_F32, torch.bfloat16: DVP_BF16, torch.float16: DVP_F16}
 _SIDE_FIELDS = ("max", "lse", "lse_safe", "logp", "logp_mp", "comp_mp", "count", "mask")
@@ -200,6 +200,8 @@ def load_library() -> ctypes.CDLL:
         lib.dvp_status_string.argtypes = [ctypes.c_int]
         lib.dvp_status_string.restype = ctypes.c_char_p
         lib.dvp_version.restype = ctypes.c_int
+        lib.dvp_row_wait_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
+        lib.dvp_row_wait_status.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -349,6 +351,16 @@ def dvp_backward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, upst
     if st != DVP_OK:
         raise DvpError(st, "dvp_backward")
     return grad_train
+
+
+def dvp_row_wait_status() -> int:
+    """Synchronises the current device and returns (and clears) the status word of
+    the resident-row kernel: 0 unless one of its bounded waits ran out."""
+    out = ctypes.c_uint32(0)
+    st = load_library().dvp_row_wait_status(ctypes.byref(out))
+    if st != 0:
+        raise DvpError(st, "dvp_row_wait_status")
+    return int(out.value)
 
 
 def dvp_gemm_tn(a: torch.Tensor, b: torch.Tensor, *, alpha: float = 1.0, out: torch.Tensor | None = None,

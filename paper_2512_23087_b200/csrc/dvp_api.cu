@@ -11,6 +11,7 @@ bool hint_ok(uint32_t hint) {
   const uint32_t threads = hint & 0xffff, stage = (hint >> 16) & 0xff;
   if (threads != 0 && (threads % 32 != 0 || threads > 512)) return false;
   const uint32_t cluster = (hint >> 24) & 0xff;
+  if (stage == 0x11) return cluster == 0;  // the resident-row kernel: one block per row
   return (stage == 0 || stage == 2) && (cluster == 0 || cluster == 1 || cluster == 2 || cluster == 4);
 }
 
@@ -105,6 +106,11 @@ int dvp_backward(const dvp_backward_args *a) {
                                                     a->launch_hint,
                                                     static_cast<cudaStream_t>(a->stream));
   return e == cudaSuccess ? DVP_OK : DVP_ERR_CUDA;
+}
+
+int dvp_row_wait_status(uint32_t *status_out) {
+  if (!status_out) return DVP_ERR_INVALID_ARG;
+  return dvp::read_and_clear_row_status(status_out) == cudaSuccess ? DVP_OK : DVP_ERR_CUDA;
 }
 
 const char *dvp_status_string(int status) {

@@ -404,4 +404,7 @@ cudaError_t launch_row_kernels(const RowParams &p, int logits_dtype, int grad_dt
 cudaError_t launch_backward_kernel(const BackwardParams &p, int logits_dtype, int grad_dtype,
                                    uint32_t hint, cudaStream_t s);
 
+// Synchronises the current device, reads the resident-row kernel's status word and clears it.
+cudaError_t read_and_clear_row_status(uint32_t *host_out);
+
 }  // namespace dvp

@@ -11,6 +11,33 @@ cudaError_t launch_backward_kernel_f32(const BackwardParams &, int, uint32_t, cu
 cudaError_t launch_backward_kernel_bf16(const BackwardParams &, int, uint32_t, cudaStream_t);
 cudaError_t launch_backward_kernel_f16(const BackwardParams &, int, uint32_t, cudaStream_t);
 
+// Status word of the resident-row kernel: waits that ran out leave their code here.
+static __device__ unsigned int g_row_status;
+
+namespace res {
+unsigned int *row_status_word() {
+  // one address per device; the symbol exists on every device that loads the library
+  static unsigned int *cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cached[dev]) {
+    void *ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_row_status) != cudaSuccess) return nullptr;
+    cached[dev] = static_cast<unsigned int *>(ptr);
+  }
+  return cached[dev];
+}
+}  // namespace res
+
+cudaError_t read_and_clear_row_status(uint32_t *host_out) {
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return e;
+  e = cudaMemcpyFromSymbol(host_out, g_row_status, sizeof(uint32_t));
+  if (e != cudaSuccess) return e;
+  const unsigned int zero = 0;
+  return cudaMemcpyToSymbol(g_row_status, &zero, sizeof(zero));
+}
+
 cudaError_t launch_row_kernels(const RowParams &p, int logits_dtype, int grad_dtype, uint32_t hint,
                                cudaStream_t s) {
   switch (logits_dtype) {

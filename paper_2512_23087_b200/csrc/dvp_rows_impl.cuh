@@ -747,6 +747,10 @@ __global__ void dvp_backward_kernel(const BackwardParams p) {
 }
 
 
+}  // namespace dvp
+#include "dvp_rows_resident.cuh"
+namespace dvp {
+
 // ---- host-side launchers, instantiated once per logits type -------------------
 
 static inline bool aligned32(const void *base, long long ld, size_t elem) {
@@ -784,6 +788,15 @@ template <typename TIn, typename TGrad>
 static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s) {
   constexpr int kElems = Granule<TIn>::kElems;
   int threads = hint & 0xffff, stage = (hint >> 16) & 0xff, cluster = (hint >> 24) & 0xff;
+  // stage byte 0x11: the kernel that keeps the row in shared memory
+  if (stage == 0x11) {
+    const bool ok16 = aligned32(p.train, p.ld_train, sizeof(TIn)) &&
+                      aligned32(p.infer, p.ld_infer, sizeof(TIn)) &&
+                      aligned32(p.grad, p.ld_grad, sizeof(TGrad));
+    const cudaError_t e = ok16 ? res::launch_resident<TIn, TGrad>(p, s) : cudaErrorNotSupported;
+    if (e != cudaErrorNotSupported) return e;
+    cluster = 0;  // rows it cannot take: the streaming kernel below
+  }
   // measured on B200: 4-byte logits run best with 2 x 512 threads per SM, 2-byte
   // logits (twice the exponentials per byte) with 4 x 256
   if (threads == 0) threads = sizeof(TIn) == 4 ? 512 : 256;
