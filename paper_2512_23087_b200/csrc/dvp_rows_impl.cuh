@@ -151,10 +151,10 @@ __device__ __forceinline__ void store_zero_granule(TGrad *dst) {
 // Per warp, in the order (slot, lane): entry = ordinal of the granule among the
 // warp's granules.  A warp whose hot granules do not fit (a dense safe set)
 // walks all of its granules instead, which is then the efficient thing to do.
-constexpr int kHotCap = 256;
+constexpr int kHotCap = 1024;  // 16-bit entries: slot * 32 + lane stays below 65536 for every row the bounds fit
 
 struct HotList {
-  uint32_t *slots;
+  uint16_t *slots;
   int count;  // granules at or above the threshold (may exceed kHotCap)
   __device__ __forceinline__ bool fits() const { return count <= kHotCap; }
 };
@@ -165,7 +165,7 @@ struct HotList {
 // not depend on how many granules are hot, and the order of the list is fixed.
 template <int kStage>
 __device__ __forceinline__ HotList build_hot_list(const uint16_t *bound, int n_steps, float tau_b,
-                                                  uint32_t *hot_smem) {
+                                                  uint16_t *hot_smem) {
   static_assert(kStage == 2, "the packed scan reads the two bounds of a step as one word");
   const int lane = threadIdx.x & 31, tid = threadIdx.x;
   HotList h;
@@ -194,7 +194,7 @@ __device__ __forceinline__ HotList build_hot_list(const uint16_t *bound, int n_s
       const int b = __ffs(acc) - 1;
       acc &= acc - 1;
       const int slot = (step0 + (b & 15)) * 2 + (b >> 4);
-      if (pos < kHotCap) h.slots[pos] = (uint32_t)(slot * 32 + lane);
+      if (pos < kHotCap) h.slots[pos] = (uint16_t)(slot * 32 + lane);
       ++pos;
     }
     h.count += __shfl_sync(0xffffffffu, incl, 31);
@@ -386,7 +386,7 @@ __device__ __forceinline__ LogSum row_sweep1(const TIn *row, int V, uint16_t *bo
 template <typename TIn, int kStage>
 __device__ __forceinline__ SumCount row_sweep2(const TIn *row, int V, int a, float tau, float m,
                                                const uint16_t *bound, float *scratch,
-                                               uint32_t *hot_smem, HotList &hot) {
+                                               uint16_t *hot_smem, HotList &hot) {
   constexpr int kElems = Granule<TIn>::kElems;
   const int n_full = V / kElems;
   const int n_gran = (V + kElems - 1) / kElems;
@@ -429,7 +429,7 @@ template <typename TIn, int kStage, int kCluster>
 __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int off, int v_part, int a,
                                                double log_rho, int mode, float mask_value,
                                                uint16_t *bound, float *scratch, float *cl_slots,
-                                               uint32_t *hot_smem, HotList &hot, uint32_t *mask_row) {
+                                               uint16_t *hot_smem, HotList &hot, uint32_t *mask_row) {
   const LogSum part = row_sweep1<TIn, kStage>(row + off, v_part, bound, scratch);
   const LogSum all = cluster_reduce_logsum<kCluster>(part, cl_slots);
 
@@ -526,7 +526,7 @@ __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int
 // Shared-memory layout of the row kernel, in 4-byte words: 96 for the block
 // reductions, 16 for the cluster exchange, then the hot lists, then the bounds.
 __host__ __device__ inline int smem_words_fixed(int threads) {
-  return 96 + 16 + (threads / 32) * kHotCap;
+  return 96 + 16 + (threads / 32) * kHotCap / 2;
 }
 
 // kThreads / kBlocks: the launch bounds (largest block, blocks per SM) that set
@@ -536,7 +536,7 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
   extern __shared__ __align__(16) float smem[];
   float *scratch = smem;        // 96 floats for the block reductions
   float *cl_slots = smem + 96;  // 4 exchanges x 4 floats, each written once
-  uint32_t *hot_smem = reinterpret_cast<uint32_t *>(smem + 112);  // kHotCap per warp
+  uint16_t *hot_smem = reinterpret_cast<uint16_t *>(smem + 112);  // kHotCap per warp
   uint16_t *bound = reinterpret_cast<uint16_t *>(smem + smem_words_fixed(blockDim.x));
 
   constexpr int kElems = Granule<TIn>::kElems;
