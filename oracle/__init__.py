@@ -23,6 +23,8 @@ _SRC = os.path.join(_HERE, "dvp_oracle.c")
 _LIB = os.path.join(_HERE, "libdvp_oracle.so")
 
 F32, BF16, F16 = 0, 1, 2
+# kinds of token-level importance weight (dvp_oracle_token_weight)
+WEIGHT_NONE, WEIGHT_RATIO, WEIGHT_TRUNCATE, WEIGHT_MASK = 0, 1, 2, 3
 
 
 def build(force: bool = False) -> str:
@@ -81,6 +83,11 @@ class _Batch(ctypes.Structure):
         ("grad", ctypes.c_void_p),
         ("mask_t", ctypes.c_void_p),
         ("mask_i", ctypes.c_void_p),
+        ("weight_kind", ctypes.c_int32),
+        ("pad_", ctypes.c_int32),
+        ("weight_lo", ctypes.c_double),
+        ("weight_hi", ctypes.c_double),
+        ("weight", ctypes.c_void_p),
     ]
 
 
@@ -101,6 +108,8 @@ def _load():
         lib.dvp_oracle_side_grad.restype = None
         lib.dvp_oracle_log_ratio.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
         lib.dvp_oracle_log_ratio.restype = ctypes.c_double
+        lib.dvp_oracle_token_weight.argtypes = [ctypes.c_double, ctypes.c_int, ctypes.c_double, ctypes.c_double]
+        lib.dvp_oracle_token_weight.restype = ctypes.c_double
         assert lib.dvp_oracle_sizeof_side() == ctypes.sizeof(_Side) == _SIDE_DTYPE.itemsize
         assert lib.dvp_oracle_sizeof_batch() == ctypes.sizeof(_Batch)
         _lib = lib
@@ -131,6 +140,7 @@ class Result:
     log_ratio: np.ndarray | None
     grad: np.ndarray | None  # [T, V] float64
     threads: int = 1
+    weight: np.ndarray | None = None  # [T] token-level importance weights, when asked for
 
 
 def _storage(x: np.ndarray, dtype: int) -> np.ndarray:
@@ -151,11 +161,14 @@ def _side(arr: np.ndarray, mask) -> Side:
 
 def dvp_rows(train: np.ndarray, ids: np.ndarray | None, rho: float, *, dtype: int = F32,
              infer: np.ndarray | None = None, upstream: np.ndarray | None = None,
-             want_grad: bool = False, want_mask: bool = False, threads: int = 1) -> Result:
+             want_grad: bool = False, want_mask: bool = False, threads: int = 1,
+             weight_kind: int = WEIGHT_NONE, weight_lo: float = 0.0, weight_hi: float = float("inf")) -> Result:
     """Run the row oracle on ``[T, V]`` logits (row stride may exceed V).
 
     ``ids`` are the sampled tokens (int64, negative = none), ``upstream`` the
-    per-token gradient g of the loss with respect to log pi^mp_train(a).
+    per-token gradient g of the loss with respect to log pi^mp_train(a).  With a
+    ``weight_kind`` the gradient row is that of ``g * w`` with ``w`` the token's
+    importance weight (``dvp_oracle_token_weight``), held constant.
     """
     lib = _load()
     if not (0.0 <= rho <= 1.0):
@@ -196,6 +209,13 @@ def dvp_rows(train: np.ndarray, ids: np.ndarray | None, rho: float, *, dtype: in
     if want_grad:
         grad = np.zeros((T, V), dtype=np.float64)
         b.grad = grad.ctypes.data
+    weight = None
+    if weight_kind != WEIGHT_NONE:
+        if infer is None:
+            raise ValueError("importance weights need the inference logits")
+        b.weight_kind, b.weight_lo, b.weight_hi = int(weight_kind), float(weight_lo), float(weight_hi)
+        weight = np.zeros(T, dtype=np.float64)
+        b.weight = weight.ctypes.data
     if want_mask:
         b.want_mask = 1
         mask_t = np.zeros((T, V), dtype=np.uint8)
@@ -211,6 +231,7 @@ def dvp_rows(train: np.ndarray, ids: np.ndarray | None, rho: float, *, dtype: in
         log_ratio=log_ratio,
         grad=grad,
         threads=used,
+        weight=weight,
     )
 
 
@@ -268,8 +289,14 @@ def dvp_fused_lmhead(hidden_bf16: np.ndarray, w_bf16: np.ndarray, infer_bf16: np
     return FusedResult(rows=rows, logits=z, d_hidden=grad @ w, d_w=grad.T @ h)
 
 
+def token_weight(log_ratio: float, kind: int, lo: float = 0.0, hi: float = float("inf")) -> float:
+    """The importance weight of one token from its log-ratio."""
+    return float(_load().dvp_oracle_token_weight(float(log_ratio), int(kind), float(lo), float(hi)))
+
+
 def dvp_rows_f64(z: np.ndarray, ids: np.ndarray, rho: float, upstream: np.ndarray | None = None,
-                 want_mask: bool = False) -> Result:
+                 want_mask: bool = False, infer: np.ndarray | None = None, weight_kind: int = WEIGHT_NONE,
+                 weight_lo: float = 0.0, weight_hi: float = float("inf")) -> Result:
     """Row oracle on float64 logits given directly (tiny cases in the tests)."""
     lib = _load()
     z = np.ascontiguousarray(z, dtype=np.float64)
@@ -280,14 +307,32 @@ def dvp_rows_f64(z: np.ndarray, ids: np.ndarray, rho: float, upstream: np.ndarra
     log_rho = float(np.log(rho)) if rho > 0 else -np.inf
     ids = np.ascontiguousarray(ids, dtype=np.int64)
     step = _SIDE_DTYPE.itemsize
+    side_i = log_ratio = weight = None
+    if infer is not None:
+        infer = np.ascontiguousarray(infer, dtype=np.float64)
+        side_i = np.zeros(T, dtype=_SIDE_DTYPE)
+        log_ratio = np.zeros(T)
+        weight = np.ones(T)
+    elif weight_kind != WEIGHT_NONE:
+        raise ValueError("importance weights need the inference logits")
     for t in range(T):
         p = side.ctypes.data + t * step
         lib.dvp_oracle_side(z.ctypes.data + t * V * 8, V, int(ids[t]), log_rho, p,
                             mask.ctypes.data + t * V if want_mask else None)
+        g = float(upstream[t]) if upstream is not None else 0.0
+        if infer is not None:
+            q = side_i.ctypes.data + t * step
+            lib.dvp_oracle_side(infer.ctypes.data + t * V * 8, V, int(ids[t]), log_rho, q, None)
+            log_ratio[t] = lib.dvp_oracle_log_ratio(p, q)
+            weight[t] = lib.dvp_oracle_token_weight(float(log_ratio[t]), int(weight_kind), float(weight_lo),
+                                                    float(weight_hi))
+            if weight_kind != WEIGHT_NONE and not np.isnan(weight[t]):
+                g = g * float(weight[t])
         if grad is not None:
-            lib.dvp_oracle_side_grad(z.ctypes.data + t * V * 8, V, int(ids[t]), float(upstream[t]), p,
+            lib.dvp_oracle_side_grad(z.ctypes.data + t * V * 8, V, int(ids[t]), g, p,
                                      grad.ctypes.data + t * V * 8)
-    return Result(train=_side(side, mask), infer=None, log_ratio=None, grad=grad)
+    return Result(train=_side(side, mask), infer=_side(side_i, None) if side_i is not None else None,
+                  log_ratio=log_ratio, grad=grad, weight=weight if weight_kind != WEIGHT_NONE else None)
 
 
 @dataclass

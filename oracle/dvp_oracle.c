@@ -185,6 +185,29 @@ double dvp_oracle_log_ratio(const oracle_side *tr, const oracle_side *inf) {
   return tr->logp_mp - inf->logp_mp;
 }
 
+/*
+ * Token-level importance weight from the per-token log-ratio r (the factor
+ * pi^mp_train(a) / pi^mp_infer(a) of the estimator of Thm. 5.3, formed as the
+ * exponential of the difference of log-probabilities, App. A protocol 4), as
+ * the comparison methods of Sec. 6 use it per token:
+ *   kind 0  no weighting, w = 1
+ *   kind 1  the plain ratio, w = e^r
+ *   kind 2  truncated importance sampling, w = min(e^r, hi)
+ *   kind 3  masked importance sampling, w = e^r if lo <= e^r <= hi, else 0
+ * r = -inf (a outside the training safe set) gives w = 0 in every kind; r = +inf
+ * (a outside the inference safe set only) gives +inf, hi and 0.  The weight is a
+ * constant of the gradient (it is "detached"): the per-token upstream gradient
+ * becomes g * w.
+ */
+double dvp_oracle_token_weight(double r, int kind, double lo, double hi) {
+  if (kind == 0) return 1.0;
+  if (isnan(r)) return NAN;
+  const double w = exp(r);
+  if (kind == 1) return w;
+  if (kind == 2) return w < hi ? w : hi;
+  return (w >= lo && w <= hi) ? w : 0.0;
+}
+
 /* ---- batch driver: rows are independent, split statically over threads -- */
 
 typedef struct {
@@ -201,6 +224,10 @@ typedef struct {
   double *log_ratio;
   double *grad;              /* [T, V] doubles or NULL                      */
   uint8_t *mask_t, *mask_i;  /* [T, V] bytes                                */
+  /* token-level importance weighting of the upstream gradient (needs infer) */
+  int32_t weight_kind, pad_;
+  double weight_lo, weight_hi;
+  double *weight;            /* [T] or NULL: the weight each row used       */
 } oracle_batch;
 
 typedef struct {
@@ -221,16 +248,25 @@ static void *oracle_rows(void *arg) {
     dvp_oracle_side(z, b->V, a, log_rho, &st,
                     b->want_mask && b->mask_t ? b->mask_t + t * b->V : NULL);
     if (b->side_t) b->side_t[t] = st;
-    if (b->grad)
-      dvp_oracle_side_grad(z, b->V, a, b->upstream ? b->upstream[t] : 0.0, &st,
-                           b->grad + t * b->V);
+    double w = 1.0;
     if (b->infer) {
       for (int64_t k = 0; k < b->V; ++k)
         z[k] = widen(b->infer, b->dtype, t * b->ld_infer + k);
       dvp_oracle_side(z, b->V, a, log_rho, &si,
                       b->want_mask && b->mask_i ? b->mask_i + t * b->V : NULL);
       if (b->side_i) b->side_i[t] = si;
-      if (b->log_ratio) b->log_ratio[t] = dvp_oracle_log_ratio(&st, &si);
+      const double r = dvp_oracle_log_ratio(&st, &si);
+      if (b->log_ratio) b->log_ratio[t] = r;
+      w = dvp_oracle_token_weight(r, b->weight_kind, b->weight_lo, b->weight_hi);
+      if (b->weight) b->weight[t] = w;
+    }
+    if (b->grad) {
+      for (int64_t k = 0; k < b->V; ++k)
+        z[k] = widen(b->train, b->dtype, t * b->ld_train + k);
+      const double g = b->upstream ? b->upstream[t] : 0.0;
+      /* a row without a sampled token has no weight (NaN) and no gradient */
+      dvp_oracle_side_grad(z, b->V, a, (b->weight_kind && !isnan(w)) ? g * w : g, &st,
+                           b->grad + t * b->V);
     }
   }
   free(z);

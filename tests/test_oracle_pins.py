@@ -423,3 +423,80 @@ def test_monitoring_quantities_against_library_routines_and_invariants():
     np.testing.assert_allclose(small[:, 0], var / 2, rtol=5e-3)
     flat = oracle.dvp_monitor(np.zeros((1, 64)), np.zeros((1, 64)))
     assert flat[0, 2] == pytest.approx(math.log(64), abs=1e-14)
+
+
+@pytest.mark.parametrize("kind,lo,hi", [(oracle.WEIGHT_RATIO, 0.0, math.inf), (oracle.WEIGHT_TRUNCATE, 0.0, 1.05),
+                                        (oracle.WEIGHT_MASK, 0.9, 1.1)])
+def test_importance_weighted_gradient_matches_autograd_with_a_detached_weight(kind, lo, hi):
+    """Thm. 5.3's estimator per token: weight pi^mp_train(a) / pi^mp_infer(a), formed as the
+    exponential of the difference of log-probabilities (App. A protocol 4) and held constant,
+    times grad log pi^mp_train(a); truncated / masked as the comparison methods of Sec. 6 do.
+    Checked against autograd of sum_t c_t * stopgrad(w_t) * log pi^mp_train(a_t)."""
+    rng = np.random.default_rng(17)
+    T, V, rho = 40, 300, 1e-3
+    z_np = _rows(rng, T, V, scale=3.0)
+    zi_np = z_np + rng.normal(size=z_np.shape) * 0.15
+    z = torch.from_numpy(z_np).requires_grad_(True)
+    zi = torch.from_numpy(zi_np)
+    c = torch.from_numpy(rng.normal(size=T))
+    ids_np = rng.integers(0, V, size=T)
+    ids_np[:30] = z_np.argsort(1)[np.arange(30), -1 - rng.integers(0, 3, size=30)]     # mostly likely tokens
+    ids = torch.from_numpy(ids_np)
+
+    def masked_logp(x):
+        with torch.no_grad():
+            pruned = x < x.max(dim=-1, keepdim=True).values + math.log(rho)
+        return torch.log_softmax(torch.where(pruned, torch.tensor(-math.inf, dtype=x.dtype), x), -1)[torch.arange(T), ids]
+
+    lt, li = masked_logp(z), masked_logp(zi)
+    with torch.no_grad():
+        ratio = torch.exp(lt - li)                       # +inf when only the inference side pruned a
+        ratio = torch.where(torch.isfinite(lt), ratio, torch.zeros_like(ratio))   # ratio zero when train pruned a
+        if kind == oracle.WEIGHT_TRUNCATE:
+            w = torch.clamp(ratio, max=hi)
+        elif kind == oracle.WEIGHT_MASK:
+            w = torch.where((ratio >= lo) & (ratio <= hi), ratio, torch.zeros_like(ratio))
+        else:
+            w = ratio
+    live = torch.isfinite(lt) & torch.isfinite(w) & (w != 0)
+    (c[live] * w[live] * lt[live]).sum().backward()
+    res = oracle.dvp_rows_f64(z_np, ids_np, rho, upstream=c.numpy(), infer=zi_np, weight_kind=kind,
+                              weight_lo=lo, weight_hi=hi)
+    fin = np.isfinite(w.numpy())
+    np.testing.assert_allclose(res.weight[fin], w.numpy()[fin], rtol=1e-12, atol=0)
+    assert np.array_equal(np.isinf(res.weight), np.isinf(w.numpy()))
+    rows = live.numpy() | (w.numpy() == 0) | ~np.isfinite(lt.detach().numpy())
+    np.testing.assert_allclose(res.grad[rows], z.grad.numpy()[rows], atol=1e-13, rtol=1e-11)
+    assert (res.grad[w.numpy() == 0] == 0).all()
+    # the three kinds really differ on this batch
+    assert (ratio > 1.05).any() and (ratio < 0.9).any() and live.sum() >= 10
+
+
+def test_importance_weight_closed_forms_and_pruned_tokens():
+    W = oracle.token_weight
+    assert W(0.0, oracle.WEIGHT_NONE) == 1.0 and W(-3.0, oracle.WEIGHT_NONE) == 1.0
+    assert W(0.0, oracle.WEIGHT_RATIO) == 1.0
+    assert W(math.log(2.0), oracle.WEIGHT_RATIO) == pytest.approx(2.0, rel=1e-15)
+    assert W(math.log(2.0), oracle.WEIGHT_TRUNCATE, 0.0, 1.5) == 1.5
+    assert W(math.log(0.5), oracle.WEIGHT_TRUNCATE, 0.0, 1.5) == pytest.approx(0.5, rel=1e-15)
+    assert W(math.log(2.0), oracle.WEIGHT_MASK, 0.5, 1.5) == 0.0
+    assert W(math.log(1.25), oracle.WEIGHT_MASK, 0.5, 1.5) == pytest.approx(1.25, rel=1e-15)
+    assert W(math.log(0.25), oracle.WEIGHT_MASK, 0.5, 1.5) == 0.0
+    # a outside the training safe set: ratio zero (remark after Thm. 5.3) in every kind
+    for kind in (oracle.WEIGHT_RATIO, oracle.WEIGHT_TRUNCATE, oracle.WEIGHT_MASK):
+        assert W(-math.inf, kind, 0.5, 1.5) == 0.0
+    # a outside the inference safe set only: unbounded ratio
+    assert W(math.inf, oracle.WEIGHT_RATIO) == math.inf
+    assert W(math.inf, oracle.WEIGHT_TRUNCATE, 0.0, 1.5) == 1.5
+    assert W(math.inf, oracle.WEIGHT_MASK, 0.5, 1.5) == 0.0
+    # identical policies: every weight is one, the weighted gradient is the plain one
+    rng = np.random.default_rng(3)
+    z = _rows(rng, 6, 64)
+    ids = z.argmax(1)
+    g = rng.normal(size=6)
+    plain = oracle.dvp_rows_f64(z, ids, 1e-2, upstream=g, infer=z.copy())
+    weighted = oracle.dvp_rows_f64(z, ids, 1e-2, upstream=g, infer=z.copy(), weight_kind=oracle.WEIGHT_RATIO)
+    assert (weighted.weight == 1.0).all() and np.array_equal(plain.grad, weighted.grad)
+    off = oracle.dvp_rows_f64(z, ids, 1e-2, upstream=g, infer=z.copy(), weight_kind=oracle.WEIGHT_MASK,
+                              weight_lo=1.5, weight_hi=2.0)
+    assert (off.weight == 0.0).all() and (off.grad == 0.0).all()
