@@ -81,6 +81,27 @@ enum { DVP_MODE_FINITE_MASK = 1, DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE = 2 };
 enum { DVP_ENTRY_FORWARD = 0, DVP_ENTRY_BACKWARD = 1, DVP_ENTRY_FUSED_LMHEAD = 2 };
 
 /*
+ * `weight_kind` of dvp_forward_args: the per-token upstream gradient is
+ * multiplied inside the kernel by a token-level importance weight w_t formed
+ * from the token's own log-ratio r_t = ln pi^mp_train(a_t) - ln pi^mp_infer(a_t)
+ * (the per-token factor of the estimator of Thm. 5.3, computed as the
+ * exponential of a difference of log-probabilities, App. A protocol 4) and held
+ * constant, so that one call gives the gradient of
+ * sum_t upstream_t * stopgrad(w_t) * ln pi^mp_train(a_t):
+ *   DVP_WEIGHT_NONE      w = 1 (upstream is used as given)
+ *   DVP_WEIGHT_RATIO     w = e^r
+ *   DVP_WEIGHT_TRUNCATE  w = min(e^r, weight_hi)      (truncated importance sampling)
+ *   DVP_WEIGHT_MASK      w = e^r if weight_lo <= e^r <= weight_hi, else 0
+ *                                                      (masked importance sampling)
+ * r = -inf (a outside V_S) gives w = 0; r = +inf (a outside V'_S only) gives
+ * +inf, weight_hi and 0.  Sec. 6 names the two comparison methods and "a
+ * threshold of 0.2" without saying what it bounds: the bounds are the caller's.
+ * Sequence-level weights (the product over a trajectory) and the token veto need
+ * every token of the sequence first: use dvp_sequence_aggregate and dvp_backward.
+ */
+enum { DVP_WEIGHT_NONE = 0, DVP_WEIGHT_RATIO = 1, DVP_WEIGHT_TRUNCATE = 2, DVP_WEIGHT_MASK = 3 };
+
+/*
  * Per-token outputs of one policy ("side"): each pointer is a device array of
  * T elements and may be NULL when the caller does not want it.
  */
@@ -114,6 +135,10 @@ typedef struct {
  *                 -inf when a is outside V_S (importance ratio zero, remark
  *                 after Thm. 5.3), +inf when a is in V_S but outside V'_S
  *   flags         device [T] bytes, DVP_FLAG_* bits
+ *   weight_kind   DVP_WEIGHT_*; other than NONE needs infer_logits, upstream and
+ *                 grad_train; weight_lo <= weight_hi, both >= 0, not NaN
+ *   weight_out    device [T] float32 or NULL: the weight each token used (NaN
+ *                 for a row without a valid sampled id)
  *   launch_hint   0 = library default; otherwise threads per block (a multiple
  *                 of 32, at most 512) in the low 16 bits, 0 or 2 in the next 8
  *                 bits, and the number of blocks that share one row (0, 1, 2 or
@@ -150,7 +175,9 @@ typedef struct {
   uint32_t launch_hint;
   uint32_t mode;      /* DVP_MODE_* bits */
   float mask_value;   /* used with DVP_MODE_FINITE_MASK */
-  uint32_t reserved_;
+  uint32_t weight_kind; /* DVP_WEIGHT_* */
+  float weight_lo, weight_hi;
+  float *weight_out;
 } dvp_forward_args;
 
 int dvp_forward(const dvp_forward_args *args);

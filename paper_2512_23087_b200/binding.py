@@ -23,6 +23,7 @@ DVP_FLAG_IN_TRAIN, DVP_FLAG_IN_INFER, DVP_FLAG_NO_ID, DVP_FLAG_BAD_ID = 1, 2, 64
 DVP_ENTRY_FORWARD, DVP_ENTRY_BACKWARD, DVP_ENTRY_FUSED_LMHEAD = 0, 1, 2
 DVP_STATIC_WORKSPACE_BYTES = 32 * 1024 * 1024
 DVP_MODE_FINITE_MASK, DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE = 1, 2
+DVP_WEIGHT_NONE, DVP_WEIGHT_RATIO, DVP_WEIGHT_TRUNCATE, DVP_WEIGHT_MASK = 0, 1, 2, 3
 
 EXPORTS = ("dvp_forward", "dvp_backward", "dvp_fused_lmhead_forward_backward",
            "dvp_fused_lmhead_forward_backward_static", "dvp_sequence_aggregate", "dvp_monitor", "dvp_gemm_tn",
@@ -67,7 +68,10 @@ class ForwardArgs(ctypes.Structure):
         ("launch_hint", ctypes.c_uint32),
         ("mode", ctypes.c_uint32),
         ("mask_value", ctypes.c_float),
-        ("reserved_", ctypes.c_uint32),
+        ("weight_kind", ctypes.c_uint32),
+        ("weight_lo", ctypes.c_float),
+        ("weight_hi", ctypes.c_float),
+        ("weight_out", ctypes.c_void_p),
     ]
 
 
@@ -249,7 +253,8 @@ def dvp_forward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, *,
                 infer_logits: torch.Tensor | None = None, upstream: torch.Tensor | None = None,
                 grad_train: torch.Tensor | None = None, grad_dtype: torch.dtype | None = None,
                 want_mask: bool = False, stream=None, launch_hint: int = 0, out=None,
-                mask_value: float | None = None, threshold_in_logits_dtype: bool = False):
+                mask_value: float | None = None, threshold_in_logits_dtype: bool = False,
+                weight_kind: int = DVP_WEIGHT_NONE, weight_lo: float = 0.0, weight_hi: float = float("inf")):
     """Pruned log-probabilities of the sampled tokens for the training and the
     inference logits (Def. 5.1, Def. 5.2), their log-ratio, and, when
     ``upstream`` is given, dLoss/dlogits (Prop. 5.4) in the same launch.
@@ -257,6 +262,10 @@ def dvp_forward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, *,
     ``mask_value`` (finite) switches to the App. A listing's semantics: pruned
     logits are replaced by it instead of by -inf; ``threshold_in_logits_dtype``
     rounds the threshold the way an eager tensor expression would.
+    ``weight_kind`` (``DVP_WEIGHT_*``) multiplies each token's upstream gradient
+    inside the kernel by the token's importance weight e^{log_ratio}, plain,
+    truncated at ``weight_hi`` or masked outside [``weight_lo``, ``weight_hi``]
+    (Thm. 5.3 per token); the weights used come back as ``weight``.
 
     Returns a namespace with ``train`` / ``infer`` (per-token tensors),
     ``log_ratio``, ``flags`` and ``grad_train``.  Pass the namespace of an
@@ -310,6 +319,12 @@ def dvp_forward(train_logits: torch.Tensor, ids: torch.Tensor, rho: float, *,
     a.mode = (DVP_MODE_FINITE_MASK if mask_value is not None else 0) | \
         (DVP_MODE_THRESHOLD_IN_LOGITS_DTYPE if threshold_in_logits_dtype else 0)
     a.mask_value = float(mask_value) if mask_value is not None else 0.0
+    a.weight_kind = int(weight_kind)
+    a.weight_lo, a.weight_hi = float(weight_lo), float(weight_hi)
+    if weight_kind != DVP_WEIGHT_NONE:
+        if getattr(res, "weight", None) is None:
+            res.weight = torch.empty(T, dtype=torch.float32, device=dev)
+        a.weight_out = _ptr(res.weight)
     st = lib.dvp_forward(ctypes.byref(a))
     if st != DVP_OK:
         raise DvpError(st, "dvp_forward")

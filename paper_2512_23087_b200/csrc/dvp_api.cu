@@ -46,6 +46,13 @@ int dvp_forward(const dvp_forward_args *a) {
   if (!a->infer_logits && (!side_empty(a->infer) || a->log_ratio)) return DVP_ERR_INVALID_ARG;
   if ((a->upstream != nullptr) != (a->grad_train != nullptr)) return DVP_ERR_INVALID_ARG;
   if (a->grad_train && (a->ld_grad < a->V || !a->ids)) return DVP_ERR_INVALID_ARG;
+  if (a->weight_kind > DVP_WEIGHT_MASK) return DVP_ERR_INVALID_ARG;
+  if (a->weight_kind != DVP_WEIGHT_NONE) {
+    if (!a->infer_logits || !a->grad_train) return DVP_ERR_INVALID_ARG;
+    if (!(a->weight_lo >= 0.f && a->weight_hi >= a->weight_lo)) return DVP_ERR_INVALID_ARG;
+  } else if (a->weight_out) {
+    return DVP_ERR_INVALID_ARG;
+  }
 
   dvp::RowParams p{};
   p.train = a->train_logits;
@@ -66,6 +73,10 @@ int dvp_forward(const dvp_forward_args *a) {
   p.out_i = a->infer;
   p.log_ratio = a->log_ratio;
   p.flags = a->flags;
+  p.weight_kind = (int)a->weight_kind;
+  p.weight_lo = a->weight_lo;
+  p.weight_hi = a->weight_hi;
+  p.weight_out = a->weight_out;
   const cudaError_t e = dvp::launch_row_kernels(p, a->logits_dtype, a->grad_dtype, a->launch_hint,
                                                 static_cast<cudaStream_t>(a->stream));
   return e == cudaSuccess ? DVP_OK : DVP_ERR_CUDA;

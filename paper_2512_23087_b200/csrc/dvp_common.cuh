@@ -298,6 +298,9 @@ struct RowParams {
   dvp_side_out out_t, out_i;
   float *log_ratio;
   uint8_t *flags;
+  int weight_kind;  // DVP_WEIGHT_*: the upstream gradient is multiplied by the token's importance weight
+  float weight_lo, weight_hi;
+  float *weight_out;
 };
 
 __device__ __forceinline__ long long load_id(const void *ids, int is_i32, long long t) {
@@ -346,6 +349,14 @@ __device__ __forceinline__ void set_mask_mass(SideStats &st, long long V, int mo
   st.live = has_a && (st.member || (mode & DVP_MODE_FINITE_MASK));
 }
 
+// ln pi^mp(a) of a row with a valid sampled token, exactly as finish_side writes it.
+__device__ __forceinline__ float logp_mp_of(const SideStats &st) {
+  const float log_ss = logf(st.s_x + st.e_a + st.s_mask);
+  if (st.member) return (st.z_a - st.m) - log_ss;
+  if (st.e_mask > 0.f) return logf(st.e_mask) - log_ss;  // a masked token keeps the mask value's probability
+  return kNegInf;
+}
+
 // Writes the per-token outputs of one side; called by one thread.
 __device__ __forceinline__ float finish_side(const dvp_side_out &o, long long t, const SideStats &st,
                                              bool has_id, bool bad_id) {
@@ -355,14 +366,12 @@ __device__ __forceinline__ float finish_side(const dvp_side_out &o, long long t,
   float logp = nan, logp_mp = nan, comp = nan;
   if (has_id) {
     logp = (float)((double)st.z_a - st.lse);
+    logp_mp = logp_mp_of(st);
     if (st.member) {
-      logp_mp = (st.z_a - st.m) - log_ss;
       comp = (st.s_x + st.s_mask) / s_tot;
-    } else if (st.e_mask > 0.f) {  // a masked token keeps the mask value's probability
-      logp_mp = logf(st.e_mask) - log_ss;
+    } else if (st.e_mask > 0.f) {
       comp = (s_tot - st.e_mask) / s_tot;
     } else {
-      logp_mp = kNegInf;
       comp = 1.f;
     }
   }
@@ -382,6 +391,27 @@ __device__ __forceinline__ float log_ratio_of(bool in_train, bool in_infer, floa
   if (!in_train) return kNegInf;
   if (!in_infer) return -kNegInf;
   return lt - li;
+}
+
+// Token-level importance weight from the log-ratio r (DVP_WEIGHT_*): the per-token
+// factor of the estimator of Thm. 5.3, optionally truncated or masked.
+__device__ __forceinline__ float token_weight(float r, int kind, float lo, float hi) {
+  if (kind == DVP_WEIGHT_NONE) return 1.f;
+  if (r != r) return r;
+  const float w = expf(r);  // e^{-inf} = 0, e^{+inf} = +inf
+  if (kind == DVP_WEIGHT_RATIO) return w;
+  if (kind == DVP_WEIGHT_TRUNCATE) return fminf(w, hi);
+  return (w >= lo && w <= hi) ? w : 0.f;
+}
+
+// The weight of row t from the statistics of both sides (every thread computes the
+// same value), NaN without a valid sampled token.
+__device__ __forceinline__ float row_weight(const RowParams &p, const SideStats &st, const SideStats &si,
+                                            bool valid_id) {
+  if (!valid_id) return __int_as_float(0x7fc00000);
+  const float lt = logp_mp_of(st), li = logp_mp_of(si);
+  const float r = (p.mode & DVP_MODE_FINITE_MASK) ? lt - li : log_ratio_of(st.member, si.member, lt, li);
+  return token_weight(r, p.weight_kind, p.weight_lo, p.weight_hi);
 }
 
 // Arguments of the stand-alone backward map.

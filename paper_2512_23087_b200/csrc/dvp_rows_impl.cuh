@@ -553,34 +553,43 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
   const int v_part = max(0, min(V - off, per_rank * kElems));
 
   const TIn *trow = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
+  const TIn *irow = p.infer ? reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer : nullptr;
   uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * ((p.V + 31) / 32) : nullptr;
-  HotList hot;
-  const SideStats st =
-      row_stats<TIn, kStage, kCluster>(trow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value, bound,
-                                       scratch, cl_slots, hot_smem, hot, mask_t);
+  uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
+  // with an importance weight the gradient needs the inference side's result first
+  const bool infer_first = p.weight_kind != DVP_WEIGHT_NONE && irow != nullptr;
+  HotList hot, hot_i;
+  SideStats st, si;
+  float w = 1.f;
+  if (infer_first) {
+    si = row_stats<TIn, kStage, kCluster>(irow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value, bound,
+                                          scratch, cl_slots + 8, hot_smem, hot_i, mask_i);
+    __syncthreads();  // the bounds and the hot lists are reused for the second matrix
+  }
+  st = row_stats<TIn, kStage, kCluster>(trow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value, bound,
+                                        scratch, cl_slots, hot_smem, hot, mask_t);
+  if (infer_first) w = row_weight(p, st, si, a >= 0);
 
   if (p.grad) {
-    const float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
+    float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
+    if (infer_first && w == w) g *= w;
     const int a_part = (a >= off && a < off + v_part) ? a - off : -1;
     row_grad<TIn, TGrad, kStage>(trow + off, reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad + off,
                                  v_part, a_part, st, g, bound, hot);
   }
 
-  SideStats si;
-  if (p.infer) {
+  if (irow && !infer_first) {
     __syncthreads();  // the bounds and the hot lists are reused for the second matrix
-    const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
-    uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
-    HotList hot_i;
     si = row_stats<TIn, kStage, kCluster>(irow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value,
                                           bound, scratch, cl_slots + 8, hot_smem, hot_i, mask_i);
   }
+  if (p.weight_out && threadIdx.x == 0 && rank == 0) p.weight_out[t] = w;
 
   if (threadIdx.x == 0 && rank == 0) {
     const float lt = finish_side(p.out_t, t, st, has_id, bad_id);
     uint8_t flags = (uint8_t)((st.member ? DVP_FLAG_IN_TRAIN : 0) | (has_id ? 0 : DVP_FLAG_NO_ID) |
                               (bad_id ? DVP_FLAG_BAD_ID : 0));
-    if (p.infer) {
+    if (irow) {
       const float li = finish_side(p.out_i, t, si, has_id, bad_id);
       if (si.member) flags |= DVP_FLAG_IN_INFER;
       if (p.log_ratio)
@@ -652,13 +661,21 @@ __global__ void dvp_row_kernel_scalar(const RowParams p) {
   const long long a = (has_id && !bad_id) ? id : -1;
 
   const TIn *trow = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
+  const TIn *irow = p.infer ? reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer : nullptr;
   uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * ((p.V + 31) / 32) : nullptr;
+  uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
   const SideStats st =
       row_stats_scalar<TIn>(trow, p.V, a, p.log_rho, p.mode, p.mask_value, scratch, mask_t);
+  SideStats si;
+  if (irow) si = row_stats_scalar<TIn>(irow, p.V, a, p.log_rho, p.mode, p.mask_value, scratch, mask_i);
+  float w = 1.f;
+  if (p.weight_kind != DVP_WEIGHT_NONE && irow) w = row_weight(p, st, si, a >= 0);
+  if (p.weight_out && threadIdx.x == 0) p.weight_out[t] = w;
 
   if (p.grad) {
     TGrad *grow = reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad;
-    const float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
+    float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
+    if (w == w) g *= w;
     const float s_tot = st.s_x + st.e_a + st.s_mask;
     const bool live = st.live;
     const float coef = live ? -g / s_tot : 0.f;
@@ -669,13 +686,6 @@ __global__ void dvp_row_kernel_scalar(const RowParams p) {
       if (live && st.member && k == a) out = g_a;
       grow[k] = Storage<TGrad>::narrow(out);
     }
-  }
-
-  SideStats si;
-  if (p.infer) {
-    const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
-    uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
-    si = row_stats_scalar<TIn>(irow, p.V, a, p.log_rho, p.mode, p.mask_value, scratch, mask_i);
   }
 
   if (threadIdx.x == 0) {

@@ -412,7 +412,8 @@ __device__ __forceinline__ void grad_vector(const uint4 &r, TGrad *dst, const Pa
 template <typename TIn, typename TGrad>
 __device__ __forceinline__ SideStats consume_side(const TIn *row, TGrad *grow, float g, int V, int a,
                                                   const RowParams &p, Walk &wk, Reducer &red,
-                                                  uint32_t *mask_row) {
+                                                  uint32_t *mask_row, const SideStats *other = nullptr,
+                                                  float *weight = nullptr) {
   constexpr int kElems = Vec<TIn>::kElems;
   using PT = PackedTau<TIn>;
   const int tid = threadIdx.x, lane = tid & 31;
@@ -550,6 +551,11 @@ __device__ __forceinline__ SideStats consume_side(const TIn *row, TGrad *grow, f
   // a safe token are zeros and need no read; the flagged ones are read again from
   // their resident slot, or from global memory (L2) when they were streamed.
   const int n_res = wk.geo.n_chunks - wk.geo.n_stream;
+  if (other) {  // the importance weight of this token, from both sides' statistics
+    const float wt = row_weight(p, st, *other, has_a);
+    *weight = wt;
+    if (wt == wt) g *= wt;
+  }
   if (has_grad) {
     const float s_tot = st.s_x + st.e_a + st.s_mask;
     const bool live = st.live;
@@ -606,6 +612,8 @@ __global__ void __launch_bounds__(kThreads, 1) dvp_row_kernel_resident(const Res
   const Geometry geo = rp.geo;
   const int V = (int)p.V;
   const bool two_sides = p.infer != nullptr;
+  // with an importance weight the gradient needs the inference side's result first
+  const bool infer_first = two_sides && p.weight_kind != DVP_WEIGHT_NONE;
   const int n_slots = geo.res_slots + geo.str_slots;
 
   if (threadIdx.x == 0) {
@@ -643,8 +651,9 @@ __global__ void __launch_bounds__(kThreads, 1) dvp_row_kernel_resident(const Res
       };
       for (long long t = blockIdx.x; t < p.T && ok; t += gridDim.x) {
         for (int side = 0; side < (two_sides ? 2 : 1) && ok; ++side) {
-          const TIn *row = side == 0 ? reinterpret_cast<const TIn *>(p.train) + t * p.ld_train
-                                     : reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
+          const bool train_side = (side == 0) != infer_first;
+          const TIn *row = train_side ? reinterpret_cast<const TIn *>(p.train) + t * p.ld_train
+                                      : reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
           const char *src = reinterpret_cast<const char *>(row);
           for (int ch = 0; ch < geo.n_stream && ok; ++ch)  // sweep 1, streamed part
             ok = issue(src, ch, str, geo.res_slots, geo.str_slots);
@@ -671,16 +680,23 @@ __global__ void __launch_bounds__(kThreads, 1) dvp_row_kernel_resident(const Res
       const int a = (has_id && !bad_id) ? (int)id : -1;
 
       const TIn *trow = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
+      const TIn *irow = two_sides ? reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer : nullptr;
       TGrad *grow = p.grad ? reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad : nullptr;
       const float g = p.grad ? p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f) : 0.f;
       uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * mask_words : nullptr;
-      const SideStats st = consume_side<TIn, TGrad>(trow, grow, g, V, a, p, wk, red, mask_t);
-      SideStats si;
-      if (two_sides) {
-        const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
-        uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * mask_words : nullptr;
+      uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * mask_words : nullptr;
+      SideStats st, si;
+      float wgt = 1.f;
+      if (infer_first) {
         si = consume_side<TIn, TGrad>(irow, (TGrad *)nullptr, 0.f, V, a, p, wk, red, mask_i);
+        // sweep 3 needs the weight between sweeps 2 and 3 of the training side: the callee
+        // forms it from both sides' statistics
+        st = consume_side<TIn, TGrad>(trow, grow, g, V, a, p, wk, red, mask_t, &si, &wgt);
+      } else {
+        st = consume_side<TIn, TGrad>(trow, grow, g, V, a, p, wk, red, mask_t);
+        if (two_sides) si = consume_side<TIn, TGrad>(irow, (TGrad *)nullptr, 0.f, V, a, p, wk, red, mask_i);
       }
+      if (p.weight_out && threadIdx.x == 0 && !ctl->abort) p.weight_out[t] = wgt;
       if (threadIdx.x == 0 && !ctl->abort) {
         const float lt = finish_side(p.out_t, t, st, has_id, bad_id);
         uint8_t flags = (uint8_t)((st.member ? DVP_FLAG_IN_TRAIN : 0) | (has_id ? 0 : DVP_FLAG_NO_ID) |

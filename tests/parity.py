@@ -9,6 +9,10 @@ Tolerances (stated once, used by every parity test):
     and NaNs must coincide;
   * lse, lse_safe: 1e-4 absolute plus one float32 rounding of the value (they
     are float32 outputs whose magnitude can reach the hundreds);
+  * importance weights (weight_kind): 2e-4 relative (two log-probabilities of
+    1e-4 each in the exponent), infinities and NaNs must coincide; rows whose
+    ratio lies within 5e-4 relative of a masking bound, where the weight jumps,
+    are counted and left out of the weight and gradient comparison;
   * gradients: per row, ||G - G_oracle||_2 <= (1e-3 + u) ||G_oracle||_2 with u
     the unit roundoff of the gradient's storage type (0 for float32, 2^-8 for
     bfloat16, 2^-11 for float16): round-to-nearest storage alone contributes
@@ -39,13 +43,14 @@ def to_oracle_storage(x: torch.Tensor) -> np.ndarray:
     return x.view(torch.int16).numpy().view(np.uint16)
 
 
-def run_oracle(train, infer, ids, rho, upstream=None, want_mask=False, threads=8):
+def run_oracle(train, infer, ids, rho, upstream=None, want_mask=False, threads=8, weight=None):
+    kw = {} if weight is None else dict(weight_kind=weight[0], weight_lo=weight[1], weight_hi=weight[2])
     return oracle.dvp_rows(
         to_oracle_storage(train), ids.detach().cpu().numpy().astype(np.int64), rho,
         dtype=ORACLE_DTYPE[train.dtype],
         infer=to_oracle_storage(infer) if infer is not None else None,
         upstream=upstream.detach().cpu().numpy().astype(np.float64) if upstream is not None else None,
-        want_grad=upstream is not None, want_mask=want_mask, threads=threads)
+        want_grad=upstream is not None, want_mask=want_mask, threads=threads, **kw)
 
 
 def near_threshold_rows(stored: torch.Tensor, side) -> np.ndarray:
@@ -158,4 +163,28 @@ def check_forward(res_gpu, batch, rho, V, want_grad, report=None, threads=8):
         check_grad(res_gpu.grad_train, want.grad, report)
     report["mean_safe_set_size"] = float(want.train.count.mean())
     report["frac_sampled_in_train_set"] = float(want.train.member.mean())
+    return report, want
+
+
+def check_weighted(res_gpu, batch, rho, V, weight, report=None, threads=8):
+    """dvp_forward with an in-kernel importance weight against the oracle's weighted gradient."""
+    report = {} if report is None else report
+    kind, lo, hi = weight
+    want = run_oracle(batch.train, batch.infer, batch.ids, rho, upstream=batch.upstream, threads=threads,
+                      weight=weight)
+    ratio = np.exp(want.log_ratio)
+    near = np.zeros(len(ratio), dtype=bool)
+    if kind == oracle.WEIGHT_MASK:
+        with np.errstate(invalid="ignore"):
+            near = (np.abs(ratio - lo) <= 5e-4 * lo) | (np.abs(ratio - hi) <= 5e-4 * hi)
+    ok = ~near
+    report["near_weight_bound_rows"] = int(near.sum())
+    report["weight_err"] = _close(res_gpu.weight.cpu(), want.weight, lambda w: 2e-4 * np.abs(w), "weight", ok)
+    # an unbounded plain ratio (token pruned on the inference side only) has no finite gradient row
+    unbounded = np.isinf(want.weight)
+    report["unbounded_weight_rows"] = int(unbounded.sum())
+    ok = ok & ~unbounded
+    check_grad(res_gpu.grad_train, want.grad, report, rows=ok, label="weighted_grad")
+    report["zero_weight_rows"] = int((want.weight[ok] == 0).sum())
+    report["live_rows"] = int(((want.weight[ok] != 0) & (want.train.member[ok] == 1)).sum())
     return report, want
