@@ -531,7 +531,10 @@ __host__ __device__ inline int smem_words_fixed(int threads) {
 
 // kThreads / kBlocks: the launch bounds (largest block, blocks per SM) that set
 // the register budget of this instantiation.  kCluster blocks share one row.
-template <typename TIn, typename TGrad, int kStage, int kThreads, int kBlocks, int kCluster>
+// kWeighted: the upstream gradient is multiplied by the token's importance weight, which
+// needs the inference side's statistics before sweep 3 of the training row: that
+// instantiation sweeps the inference row first.
+template <typename TIn, typename TGrad, int kStage, int kThreads, int kBlocks, int kCluster, bool kWeighted>
 __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowParams p) {
   extern __shared__ __align__(16) float smem[];
   float *scratch = smem;        // 96 floats for the block reductions
@@ -553,43 +556,48 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
   const int v_part = max(0, min(V - off, per_rank * kElems));
 
   const TIn *trow = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
-  const TIn *irow = p.infer ? reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer : nullptr;
   uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * ((p.V + 31) / 32) : nullptr;
-  uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
-  // with an importance weight the gradient needs the inference side's result first
-  const bool infer_first = p.weight_kind != DVP_WEIGHT_NONE && irow != nullptr;
-  HotList hot, hot_i;
+  HotList hot;
   SideStats st, si;
-  float w = 1.f;
-  if (infer_first) {
+  if constexpr (kWeighted) {  // the launcher guarantees an inference matrix
+    const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
+    uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
+    HotList hot_i;
     si = row_stats<TIn, kStage, kCluster>(irow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value, bound,
                                           scratch, cl_slots + 8, hot_smem, hot_i, mask_i);
     __syncthreads();  // the bounds and the hot lists are reused for the second matrix
   }
   st = row_stats<TIn, kStage, kCluster>(trow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value, bound,
                                         scratch, cl_slots, hot_smem, hot, mask_t);
-  if (infer_first) w = row_weight(p, st, si, a >= 0);
 
   if (p.grad) {
     float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
-    if (infer_first && w == w) g *= w;
+    if constexpr (kWeighted) {
+      const float w = row_weight(p, st, si, a >= 0);
+      if (w == w) g *= w;
+      if (p.weight_out && threadIdx.x == 0 && rank == 0) p.weight_out[t] = w;
+    }
     const int a_part = (a >= off && a < off + v_part) ? a - off : -1;
     row_grad<TIn, TGrad, kStage>(trow + off, reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad + off,
                                  v_part, a_part, st, g, bound, hot);
   }
 
-  if (irow && !infer_first) {
-    __syncthreads();  // the bounds and the hot lists are reused for the second matrix
-    si = row_stats<TIn, kStage, kCluster>(irow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value,
-                                          bound, scratch, cl_slots + 8, hot_smem, hot_i, mask_i);
+  if constexpr (!kWeighted) {
+    if (p.infer) {
+      __syncthreads();  // the bounds and the hot lists are reused for the second matrix
+      const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
+      uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
+      HotList hot_i;
+      si = row_stats<TIn, kStage, kCluster>(irow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value,
+                                            bound, scratch, cl_slots + 8, hot_smem, hot_i, mask_i);
+    }
   }
-  if (p.weight_out && threadIdx.x == 0 && rank == 0) p.weight_out[t] = w;
 
   if (threadIdx.x == 0 && rank == 0) {
     const float lt = finish_side(p.out_t, t, st, has_id, bad_id);
     uint8_t flags = (uint8_t)((st.member ? DVP_FLAG_IN_TRAIN : 0) | (has_id ? 0 : DVP_FLAG_NO_ID) |
                               (bad_id ? DVP_FLAG_BAD_ID : 0));
-    if (irow) {
+    if (p.infer) {
       const float li = finish_side(p.out_i, t, si, has_id, bad_id);
       if (si.member) flags |= DVP_FLAG_IN_INFER;
       if (p.log_ratio)
@@ -767,9 +775,9 @@ static inline bool aligned32(const void *base, long long ld, size_t elem) {
   return base == nullptr || (((uintptr_t)base % 32 == 0) && ((ld * (long long)elem) % 32 == 0));
 }
 
-template <typename TIn, typename TGrad, int kStage, int kThreads, int kBlocks, int kCluster>
+template <typename TIn, typename TGrad, int kStage, int kThreads, int kBlocks, int kCluster, bool kWeighted = false>
 static cudaError_t launch_rows_vec(const RowParams &p, int threads, size_t smem, cudaStream_t s) {
-  auto k = dvp_row_kernel<TIn, TGrad, kStage, kThreads, kBlocks, kCluster>;
+  auto k = dvp_row_kernel<TIn, TGrad, kStage, kThreads, kBlocks, kCluster, kWeighted>;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -816,6 +824,8 @@ static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s
                       aligned32(p.grad, p.ld_grad, sizeof(TGrad));
   const long long n_gran_row = (p.V + kElems - 1) / kElems;
   if (cluster == 0) cluster = 1;
+  const bool weighted = p.weight_kind != DVP_WEIGHT_NONE;  // one block per row only
+  if (weighted) cluster = 1;
   if (cluster > 1 && (n_gran_row < 4096 || p.T * cluster > 0x7fffffffLL)) cluster = 1;
   const long long n_gran = (n_gran_row + cluster - 1) / cluster;  // granules per block
   // shrink the block for short rows so that threads are not idle
@@ -828,6 +838,10 @@ static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s
       return launch_rows_vec<TIn, TGrad, 2, 256, 4, 4>(p, threads, smem, s);
     if (cluster == 2 && threads <= 256 && stage == 2)
       return launch_rows_vec<TIn, TGrad, 2, 256, 4, 2>(p, threads, smem, s);
+    if (weighted) {
+      if (threads > 256) return launch_rows_vec<TIn, TGrad, 2, 512, 2, 1, true>(p, threads, smem, s);
+      return launch_rows_vec<TIn, TGrad, 2, 256, 4, 1, true>(p, threads, smem, s);
+    }
     if (threads > 256) return launch_rows_vec<TIn, TGrad, 2, 512, 2, 1>(p, threads, smem, s);
     return launch_rows_vec<TIn, TGrad, 2, 256, 4, 1>(p, threads, smem, s);
   }
