@@ -349,7 +349,7 @@ __device__ __forceinline__ void set_mask_mass(SideStats &st, long long V, int mo
   st.live = has_a && (st.member || (mode & DVP_MODE_FINITE_MASK));
 }
 
-// ln pi^mp(a) of a row with a valid sampled token, exactly as finish_side writes it.
+// ln pi^mp(a) of a row with a valid sampled token, with the arithmetic of finish_side.
 __device__ __forceinline__ float logp_mp_of(const SideStats &st) {
   const float log_ss = logf(st.s_x + st.e_a + st.s_mask);
   if (st.member) return (st.z_a - st.m) - log_ss;
@@ -366,12 +366,14 @@ __device__ __forceinline__ float finish_side(const dvp_side_out &o, long long t,
   float logp = nan, logp_mp = nan, comp = nan;
   if (has_id) {
     logp = (float)((double)st.z_a - st.lse);
-    logp_mp = logp_mp_of(st);
     if (st.member) {
+      logp_mp = (st.z_a - st.m) - log_ss;
       comp = (st.s_x + st.s_mask) / s_tot;
-    } else if (st.e_mask > 0.f) {
+    } else if (st.e_mask > 0.f) {  // a masked token keeps the mask value's probability
+      logp_mp = logf(st.e_mask) - log_ss;
       comp = (s_tot - st.e_mask) / s_tot;
     } else {
+      logp_mp = kNegInf;
       comp = 1.f;
     }
   }
