@@ -142,8 +142,11 @@ typedef struct {
  *   launch_hint   0 = library default; otherwise threads per block (a multiple
  *                 of 32, at most 512) in the low 16 bits, 0 or 2 in the next 8
  *                 bits, and the number of blocks that share one row (0, 1, 2 or
- *                 4; a thread-block cluster) in the top 8 bits; tuning only, the
- *                 safe set and counts do not depend on it
+ *                 4; a thread-block cluster) in the top 8 bits.  0x11 in the
+ *                 second byte (with zero elsewhere) selects the kernel that keeps
+ *                 the row in shared memory (rows of up to 480 KB whose byte
+ *                 length is a multiple of 16; others take the default kernel).
+ *                 Tuning only: the safe set and counts do not depend on it
  *
  * Rows whose start is 32-byte aligned in all three matrices take the
  * vectorised kernels; any other layout takes a scalar kernel, same results.
@@ -403,12 +406,11 @@ int dvp_gemm_tn(const void *a, int64_t lda, const void *b, int64_t ldb, float *c
 
 /*
  * dvp_row_wait_status -- the row kernel that keeps rows resident in shared
- * memory (launch_hint stage byte 0x11 / 0x12, and the default for row shapes it
- * serves) waits on hardware barriers for its bulk copies and for the other
- * blocks of its cluster.  Every such wait is bounded; one that runs out ends the
- * launch early (outputs of that launch are then undefined) and ORs a code into a
+ * memory (launch_hint stage byte 0x11) waits on hardware barriers for its bulk
+ * copies and its block reductions.  Every such wait is bounded; one that runs
+ * out ends the launch early (its outputs are then undefined) and ORs a code into a
  * per-device status word: 1 a copy did not land, 2 a ring slot was not handed
- * back, 4 a block of the cluster did not report.  This call waits for all work
+ * back, 4 a warp did not reach a block reduction.  This call waits for all work
  * on the current device (it synchronises), copies the word to *status_out (a
  * host pointer) and clears it.  The paper has no counterpart.  0 means that no
  * wait has run out since the last call.  Errors: DVP_ERR_INVALID_ARG (NULL),

@@ -5,28 +5,30 @@
 // gradient of Prop. 5.4).  One block owns one row at a time and the second and
 // third look are served from shared memory and L2 instead of HBM:
 //
-//   * the row is cut into slots of kVec * 512 16-byte vectors.  The last R slots
-//     of a row stay in a "resident" ring of shared memory from the first sweep to
-//     the last one that needs them; the first n - R slots pass through a small
-//     "stream" ring once per sweep (the repeats come from L2: a block re-reads
-//     what it read a few microseconds earlier).  Rows of up to about 150 KB are
-//     resident as a whole.
+//   * the row is cut into slots of 30 KB (four 16-byte vectors per consumer thread).
+//     The last R slots of a row stay in a "resident" ring of shared memory from the
+//     first sweep to the last one that needs them; the first n - R slots pass
+//     through a small "stream" ring, once for sweep 1 (from HBM) and once for
+//     sweep 2 (from L2: a block re-reads what it read a few microseconds earlier).
+//     Rows of up to 120 KB are resident as a whole.
 //   * a producer warp issues every bulk copy, in the one order both sides know:
 //     per matrix ("side") of a token the streamed slots, the resident slots, the
-//     streamed slots again for sweep 2 and, with a gradient, once more for
-//     sweep 3; then the next side.  Each copy completes on its slot's "full"
-//     mbarrier and may be issued once the slot's "empty" mbarrier says that every
-//     consumer warp is done with the previous content, so the producer runs ahead
-//     of the consumers by whatever the rings have free, across sweeps, sides and
-//     tokens: the post-sweep phases (reductions, threshold, per-token results) do
-//     not interrupt the stream from HBM.
-//   * 16 consumer warps: sweep 1 (A1, A3) online log-sum-exp and maximum;
+//     streamed slots again for sweep 2; then the next side.  Each copy completes
+//     on its slot's "full" mbarrier and may be issued once the slot's "empty"
+//     mbarrier says that every consumer warp is done with the previous content,
+//     so the producer runs ahead of the consumers by whatever the rings have free,
+//     across sweeps, sides and tokens.
+//   * 15 consumer warps: sweep 1 (A1, A3) online log-sum-exp and maximum;
 //     block reduction -> threshold (A2); sweep 2 (A4) masked sum and count, only
-//     elements at or above the threshold cost more than a packed compare;
-//     block reduction -> per-token results (A5, A6); sweep 3 (A7) gradient to HBM.
+//     elements at or above the threshold cost more than a packed compare, and
+//     each thread flags its vectors that hold a safe token; block reduction ->
+//     per-token results (A5, A6); sweep 3 (A7) writes zeros for unflagged vectors
+//     without reading anything and revisits the flagged ones (resident slot, or L2).
 //
-// HBM sees each logit once and each gradient once, whatever the density of the
-// safe set.  The kernel is persistent: block b takes tokens b, b + grid, ...
+// HBM sees each logit once, whatever the density of the safe set.  Measured, it is
+// slower than the streaming kernel (one row per SM runs its phases one after
+// another); it is kept as an option behind the launch hint.  The kernel is
+// persistent: block b takes tokens b, b + grid, ...
 //
 // Every mbarrier wait is bounded.  A wait that runs out sets an abort word in
 // shared memory and a status word in global memory; from then on every wait

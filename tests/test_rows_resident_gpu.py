@@ -1,4 +1,4 @@
-"""Parity of the resident-row kernel (one block per row; the row, or its last 160 KB,
+"""Parity of the resident-row kernel (one block per row; the row, or its last 120 KB,
 stays in shared memory between the sweeps, the rest is re-read through a small
 ring) with the fp64 oracle, through the C ABI.  The kernel is selected with the
 stage byte 0x11 of ``launch_hint``."""
