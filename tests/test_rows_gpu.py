@@ -289,6 +289,30 @@ def test_full_size_sampled_rows_and_size_free_properties(name):
     parity.check_forward(sub_res, sub, rho, w.V, True)
 
 
+@pytest.mark.parametrize("rho", [1e-4, 1e-3])
+def test_full_size_forward_only_configuration(rho):
+    """T = 8192 x V = 151,936 bf16, forward only, both thresholds, as the benchmark
+    launches it: size-free properties on every row, sampled rows against the oracle."""
+    w = W["c1_bf16_fwd"]
+    batch = inputs.make_rows(w, seed=0, device=DEV)
+    T = batch.train.shape[0]
+    res = _forward(batch, rho, False, want_mask=False)
+    torch.cuda.synchronize()
+    assert res.grad_train is None
+    assert (res.train.count >= 1).all() and (res.infer.count >= 1).all()
+    member = (res.flags & 1).bool()
+    assert (res.train.logp_mp[member] <= 1e-6).all()
+    assert torch.isneginf(res.train.logp_mp[~member]).all()
+    assert (res.infer.lse_safe <= res.infer.lse + 1e-4).all()
+    both = ((res.flags & 3) == 3)
+    assert torch.isfinite(res.log_ratio[both]).all() and both.float().mean().item() > 0.8
+    pick = torch.unique(torch.cat([torch.arange(0, T, T // 32), torch.tensor([0, T - 1])])).to(DEV)
+    sub = inputs.RowBatch(batch.train[pick], batch.infer[pick], batch.ids[pick], batch.upstream[pick])
+    sub_res = type(res)(train=_take(res.train, pick), infer=_take(res.infer, pick),
+                        log_ratio=res.log_ratio[pick], flags=res.flags[pick], grad_train=None)
+    parity.check_forward(sub_res, sub, rho, w.V, False)
+
+
 def _take(side, pick):
     out = type(side)()
     for k, v in vars(side).items():
