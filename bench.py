@@ -364,7 +364,10 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
                      "kernel": "dvp_row_kernel", "bytes_per_launch": alg_bytes,
-                     "frac_of_nominal_8TBs": achieved / 8000.0},
+                     "frac_of_nominal_8TBs": achieved / 8000.0,
+                     # DRAM bytes actually moved per second against the same peak: how busy HBM is,
+                     # revisits included (None without a traffic record for these kernel sources)
+                     "dram_busy_frac": (traffic / (ms * 1e-3 / args.steps) / 1e9 / peak) if traffic else None},
     }
     if other is not None:
         if world > 1:
