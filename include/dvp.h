@@ -146,7 +146,11 @@ typedef struct {
  *                 second byte (with zero elsewhere) selects the kernel that keeps
  *                 the row in shared memory (rows of up to 480 KB whose byte
  *                 length is a multiple of 16; others take the default kernel).
- *                 Tuning only: the safe set and counts do not depend on it
+ *                 Tuning only: the safe set and counts do not depend on it.
+ *                 0x1e there is a self-test of that kernel's wait limit: its
+ *                 first block withholds its first copy, the wait for it runs out
+ *                 after about a second, the launch ends by itself with undefined
+ *                 outputs and dvp_row_wait_status reports code 1 or 2
  *
  * Rows whose start is 32-byte aligned in all three matrices take the
  * vectorised kernels; any other layout takes a scalar kernel, same results.

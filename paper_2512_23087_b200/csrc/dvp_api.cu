@@ -11,7 +11,7 @@ bool hint_ok(uint32_t hint) {
   const uint32_t threads = hint & 0xffff, stage = (hint >> 16) & 0xff;
   if (threads != 0 && (threads % 32 != 0 || threads > 512)) return false;
   const uint32_t cluster = (hint >> 24) & 0xff;
-  if (stage == 0x11) return cluster == 0;  // the resident-row kernel: one block per row
+  if (stage == 0x11 || stage == 0x1e) return cluster == 0;  // the resident-row kernel (0x1e: its self-test)
   return (stage == 0 || stage == 2) && (cluster == 0 || cluster == 1 || cluster == 2 || cluster == 4);
 }
 

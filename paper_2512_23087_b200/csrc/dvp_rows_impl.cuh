@@ -806,12 +806,14 @@ template <typename TIn, typename TGrad>
 static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s) {
   constexpr int kElems = Granule<TIn>::kElems;
   int threads = hint & 0xffff, stage = (hint >> 16) & 0xff, cluster = (hint >> 24) & 0xff;
-  // stage byte 0x11: the kernel that keeps the row in shared memory
-  if (stage == 0x11) {
+  // stage byte 0x11: the kernel that keeps the row in shared memory; 0x1e: the same with
+  // block 0's first copy withheld (self-test of the wait limit)
+  if (stage == 0x11 || stage == 0x1e) {
     const bool ok16 = aligned32(p.train, p.ld_train, sizeof(TIn)) &&
                       aligned32(p.infer, p.ld_infer, sizeof(TIn)) &&
                       aligned32(p.grad, p.ld_grad, sizeof(TGrad));
-    const cudaError_t e = ok16 ? res::launch_resident<TIn, TGrad>(p, s) : cudaErrorNotSupported;
+    const cudaError_t e =
+        ok16 ? res::launch_resident<TIn, TGrad>(p, s, stage == 0x1e) : cudaErrorNotSupported;
     if (e != cudaErrorNotSupported) return e;
     cluster = 0;  // rows it cannot take: the streaming kernel below
   }

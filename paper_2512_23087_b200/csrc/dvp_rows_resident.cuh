@@ -48,7 +48,10 @@ constexpr int kConsumerWarps = 15;
 constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kThreads = kConsumers + 32;  // + the producer warp
 constexpr int kMaxSlots = 64;
-constexpr uint32_t kSpinLimit = 1u << 22;  // x >= 40 ns once past the first polls: about a second
+// Polls of one wait.  A poll may suspend the thread for up to kSuspendNs (the hint given
+// to try_wait) and is followed by a 40 ns sleep: a wait gives up after about a second.
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSuspendNs = 200;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -67,10 +70,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(kSuspendNs)
       : "memory");
   return ok != 0;
 }
@@ -306,6 +309,7 @@ struct ResidentParams {
   RowParams row;
   Geometry geo;
   unsigned int *status;  // global status word, OR-ed with kWait* codes
+  int withhold_first;    // self-test: block 0 never issues its first copy, so its first wait runs out
 };
 
 // A slot holds kGroup 16-byte vectors per consumer thread (30 KB): one bulk copy, one
@@ -638,8 +642,14 @@ __global__ void __launch_bounds__(kThreads, 1) dvp_row_kernel_resident(const Res
       Cursor res = {0, 0}, str = {0, 0};
       bool ok = true;
       // Copies slot `ch` of a row into the next slot of a ring; false once a wait ran out.
+      bool withhold = rp.withhold_first != 0 && blockIdx.x == 0;
       auto issue = [&](const char *row_bytes, int ch, Cursor &cur, int ring_first, int ring_slots) {
         const int slot = ring_first + cur.slot;
+        if (withhold) {  // the slot is taken but nothing will ever land in it
+          withhold = false;
+          cur.advance(ring_slots);
+          return true;
+        }
         // the slot's previous use is over (a fresh barrier passes the first time round)
         if (!w.wait(smem_u32(&ctl->empty[slot]), cur.phase ^ 1, kWaitEmpty)) return false;
         if (*w.abort) return false;  // consumers no longer wait for what is issued
@@ -689,14 +699,16 @@ __global__ void __launch_bounds__(kThreads, 1) dvp_row_kernel_resident(const Res
       uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * mask_words : nullptr;
       SideStats st, si;
       float wgt = 1.f;
-      if (infer_first) {
-        si = consume_side<TIn, TGrad>(irow, (TGrad *)nullptr, 0.f, V, a, p, wk, red, mask_i);
+      // one call site for both matrices: the second copy of the sweeps would cost registers
+      for (int k = 0; k < (two_sides ? 2 : 1); ++k) {
+        const bool train_side = (k == 0) != infer_first;
         // sweep 3 needs the weight between sweeps 2 and 3 of the training side: the callee
         // forms it from both sides' statistics
-        st = consume_side<TIn, TGrad>(trow, grow, g, V, a, p, wk, red, mask_t, &si, &wgt);
-      } else {
-        st = consume_side<TIn, TGrad>(trow, grow, g, V, a, p, wk, red, mask_t);
-        if (two_sides) si = consume_side<TIn, TGrad>(irow, (TGrad *)nullptr, 0.f, V, a, p, wk, red, mask_i);
+        const SideStats r = consume_side<TIn, TGrad>(
+            train_side ? trow : irow, train_side ? grow : (TGrad *)nullptr, train_side ? g : 0.f, V, a, p, wk,
+            red, train_side ? mask_t : mask_i, (train_side && infer_first) ? &si : nullptr, &wgt);
+        if (train_side) st = r;
+        else si = r;
       }
       if (p.weight_out && threadIdx.x == 0 && !ctl->abort) p.weight_out[t] = wgt;
       if (threadIdx.x == 0 && !ctl->abort) {
@@ -748,7 +760,7 @@ static inline Geometry geometry_of(long long row_bytes) {
 }
 
 template <typename TIn, typename TGrad>
-static cudaError_t launch_resident(const RowParams &p, cudaStream_t s) {
+static cudaError_t launch_resident(const RowParams &p, cudaStream_t s, bool withhold_first = false) {
   const Geometry geo = geometry_of(p.V * (long long)sizeof(TIn));
   if (geo.n_chunks == 0) return cudaErrorNotSupported;
   auto k = dvp_row_kernel_resident<TIn, TGrad>;
@@ -764,6 +776,7 @@ static cudaError_t launch_resident(const RowParams &p, cudaStream_t s) {
   rp.row = p;
   rp.geo = geo;
   rp.status = status;
+  rp.withhold_first = withhold_first ? 1 : 0;
   const unsigned grid = (unsigned)(p.T < (long long)sms ? p.T : (long long)sms);  // one block per SM
   k<<<grid, kThreads, smem, s>>>(rp);
   return cudaGetLastError();

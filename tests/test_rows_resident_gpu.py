@@ -160,3 +160,27 @@ def test_reruns_are_bit_identical_and_agree_with_the_streaming_kernel():
     fin = torch.isfinite(other.train.logp_mp)
     assert torch.equal(fin, torch.isfinite(runs[0].train.logp_mp))
     assert (other.train.logp_mp[fin] - runs[0].train.logp_mp[fin]).abs().max().item() < 1e-5
+
+
+def test_a_wait_that_runs_out_ends_the_launch_and_is_reported():
+    """Stage byte 0x1e: block 0 of the resident-row kernel withholds its first bulk
+    copy, so the consumers' wait for it reaches its limit (about a second).  The
+    launch must end by itself, `dvp_row_wait_status` must report it once (code 1, a
+    copy did not land, or code 2, the producer found no free slot behind the stuck
+    consumers: whichever wait gives up first), and the next launch on the same
+    context must be correct."""
+    w = dataclasses.replace(W["c0_small_f32"], dtype="bf16")
+    batch = inputs.make_rows(w, seed=31, device=DEV, T=300, V=40000)
+    assert binding.dvp_row_wait_status() == 0
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    binding.dvp_forward(batch.train, batch.ids, 1e-3, infer_logits=batch.infer, upstream=batch.upstream,
+                        launch_hint=0x1e << 16)
+    t1.record()
+    status = binding.dvp_row_wait_status()          # synchronises
+    assert status in (1, 2, 3), status
+    assert t0.elapsed_time(t1) < 20000.0             # it gave up, in seconds at most
+    assert binding.dvp_row_wait_status() == 0        # the word is cleared by the read
+    res = _forward(batch, 1e-3, True, launch_hint=RESIDENT)
+    parity.check_forward(res, batch, 1e-3, 40000, True)
