@@ -249,14 +249,17 @@ class FusedResult:
 
 
 def dvp_fused_lmhead(hidden_bf16: np.ndarray, w_bf16: np.ndarray, infer_bf16: np.ndarray,
-                     ids: np.ndarray, rho: float, upstream: np.ndarray, threads: int = 1
-                     ) -> FusedResult:
+                     ids: np.ndarray, rho: float, upstream: np.ndarray, threads: int = 1,
+                     weight_kind: int = WEIGHT_NONE, weight_lo: float = 0.0,
+                     weight_hi: float = float("inf")) -> FusedResult:
     """LM-head composition: z = h W^T, then the row computation on z, then the
     chain rule of Prop. 5.6 part 2 through the linear head:
     dH = G W and dW = G^T h with G = dL/dz.
 
     hidden [T, H], w [V, H] and infer logits [T, V] are bfloat16 bit patterns
-    (uint16).  Train logits are taken in float64, so they never round.
+    (uint16).  Train logits are taken in float64, so they never round.  With a
+    ``weight_kind`` each token's upstream gradient is multiplied by its importance
+    weight (``dvp_oracle_token_weight``), held constant.
     """
     h = _bf16_bits_to_f64(hidden_bf16)
     w = _bf16_bits_to_f64(w_bf16)
@@ -274,6 +277,7 @@ def dvp_fused_lmhead(hidden_bf16: np.ndarray, w_bf16: np.ndarray, infer_bf16: np
     ids = np.ascontiguousarray(ids, dtype=np.int64)
     up = np.ascontiguousarray(upstream, dtype=np.float64)
     step = _SIDE_DTYPE.itemsize
+    weight = np.ones(T)
     for t in range(T):
         zt = np.ascontiguousarray(z[t])
         zit = np.ascontiguousarray(zi[t])
@@ -281,11 +285,16 @@ def dvp_fused_lmhead(hidden_bf16: np.ndarray, w_bf16: np.ndarray, infer_bf16: np
         pi = side_i.ctypes.data + t * step
         lib.dvp_oracle_side(zt.ctypes.data, V, int(ids[t]), log_rho, pt, None)
         lib.dvp_oracle_side(zit.ctypes.data, V, int(ids[t]), log_rho, pi, None)
-        lib.dvp_oracle_side_grad(zt.ctypes.data, V, int(ids[t]), float(up[t]), pt,
-                                 grad.ctypes.data + t * V * 8)
         log_ratio[t] = lib.dvp_oracle_log_ratio(pt, pi)
+        g = float(up[t])
+        if weight_kind != WEIGHT_NONE:
+            weight[t] = lib.dvp_oracle_token_weight(float(log_ratio[t]), int(weight_kind), float(weight_lo),
+                                                    float(weight_hi))
+            if not np.isnan(weight[t]):
+                g *= float(weight[t])
+        lib.dvp_oracle_side_grad(zt.ctypes.data, V, int(ids[t]), g, pt, grad.ctypes.data + t * V * 8)
     rows = Result(train=_side(side_t, None), infer=_side(side_i, None), log_ratio=log_ratio,
-                  grad=grad, threads=1)
+                  grad=grad, threads=1, weight=weight if weight_kind != WEIGHT_NONE else None)
     return FusedResult(rows=rows, logits=z, d_hidden=grad @ w, d_w=grad.T @ h)
 
 

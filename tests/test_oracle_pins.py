@@ -500,3 +500,42 @@ def test_importance_weight_closed_forms_and_pruned_tokens():
     off = oracle.dvp_rows_f64(z, ids, 1e-2, upstream=g, infer=z.copy(), weight_kind=oracle.WEIGHT_MASK,
                               weight_lo=1.5, weight_hi=2.0)
     assert (off.weight == 0.0).all() and (off.grad == 0.0).all()
+
+
+@pytest.mark.parametrize("kind,lo,hi", [(oracle.WEIGHT_TRUNCATE, 0.0, 1.01), (oracle.WEIGHT_MASK, 0.98, 1.05)])
+def test_weighted_fused_lmhead_matches_autograd_through_the_head(kind, lo, hi):
+    """The per-token estimator of Thm. 5.3 through a linear LM head: autograd of
+    sum_t c_t stopgrad(w_t) ln pi^mp_train(a_t) with z = h W^T gives dH and dW."""
+    rng = np.random.default_rng(31)
+    T, H, V, rho = 24, 8, 40, 2e-2
+    hb = torch.from_numpy(rng.normal(size=(T, H)).astype(np.float32)).to(torch.bfloat16)
+    wb = torch.from_numpy((rng.normal(size=(V, H)) * 0.5).astype(np.float32)).to(torch.bfloat16)
+    h = hb.to(torch.float64).requires_grad_(True)
+    w = wb.to(torch.float64).requires_grad_(True)
+    z = h @ w.t()
+    zi = (z.detach() + torch.from_numpy(rng.normal(size=(T, V)) * 0.05)).to(torch.bfloat16)
+    order = z.detach().numpy().argsort(1)
+    ids = order[np.arange(T), -1 - rng.integers(0, 2, size=T)]
+    ids[-3:] = order[np.arange(T - 3, T), 0]                     # pruned tokens
+    idt = torch.from_numpy(ids)
+    c = torch.from_numpy(rng.normal(size=T))
+
+    def masked_logp(x):
+        with torch.no_grad():
+            pruned = x < x.max(dim=-1, keepdim=True).values + math.log(rho)
+        return torch.log_softmax(torch.where(pruned, torch.tensor(-math.inf, dtype=x.dtype), x), -1)[torch.arange(T), idt]
+
+    lt, li = masked_logp(z), masked_logp(zi.to(torch.float64))
+    with torch.no_grad():
+        ratio = torch.where(torch.isfinite(lt), torch.exp(lt - li), torch.zeros_like(lt))
+        wgt = torch.clamp(ratio, max=hi) if kind == oracle.WEIGHT_TRUNCATE else \
+            torch.where((ratio >= lo) & (ratio <= hi), ratio, torch.zeros_like(ratio))
+    live = torch.isfinite(lt) & (wgt != 0)
+    (c[live] * wgt[live] * lt[live]).sum().backward()
+    bits = lambda x: x.view(torch.int16).numpy().view(np.uint16)
+    res = oracle.dvp_fused_lmhead(bits(hb), bits(wb), bits(zi), ids, rho, c.numpy(), weight_kind=kind,
+                                  weight_lo=lo, weight_hi=hi)
+    np.testing.assert_allclose(res.rows.weight, wgt.numpy(), rtol=1e-11, atol=0)
+    np.testing.assert_allclose(res.d_hidden, h.grad.numpy(), atol=1e-12)
+    np.testing.assert_allclose(res.d_w, w.grad.numpy(), atol=1e-12)
+    assert live.sum() >= 8 and (wgt == 0).sum() >= 3 and (ratio != wgt).any()
