@@ -247,6 +247,11 @@ int dvp_backward(const dvp_backward_args *args);
  *                 every tensor-core kernel finished, non-zero if one gave up
  *                 waiting (results are then invalid).
  *   panel_rows    0 = library default (at most 4096); otherwise a multiple of 128
+ *   weight_kind   DVP_WEIGHT_NONE, DVP_WEIGHT_TRUNCATE or DVP_WEIGHT_MASK, as in
+ *                 dvp_forward: each token's upstream gradient is multiplied by its
+ *                 importance weight (needs infer_logits; weight_hi must be finite,
+ *                 because the float16 gradient panel is scaled for
+ *                 max |upstream| * max(1, weight_hi)); weight_out as in dvp_forward
  *
  * ld_hidden, ld_w, ld_dh, ld_dw must be multiples of 8 and hidden, w_vocab
  * 16-byte, d_hidden, d_w 32-byte aligned (DVP_ERR_UNSUPPORTED otherwise).
@@ -278,6 +283,9 @@ typedef struct {
   void *workspace;
   size_t workspace_bytes;
   void *stream;
+  uint32_t weight_kind;
+  float weight_lo, weight_hi;
+  float *weight_out;
 } dvp_fused_args;
 
 int dvp_fused_lmhead_forward_backward(const dvp_fused_args *args);

@@ -131,6 +131,10 @@ class FusedArgs(ctypes.Structure):
         ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t),
         ("stream", ctypes.c_void_p),
+        ("weight_kind", ctypes.c_uint32),
+        ("weight_lo", ctypes.c_float),
+        ("weight_hi", ctypes.c_float),
+        ("weight_out", ctypes.c_void_p),
     ]
 
 
@@ -410,10 +414,14 @@ def dvp_fused_lmhead_forward_backward(hidden: torch.Tensor, w_vocab: torch.Tenso
                                       infer_logits: torch.Tensor | None = None,
                                       d_w: torch.Tensor | None = None, accumulate_dw: bool = False,
                                       panel_rows: int = 0, workspace: torch.Tensor | None = None,
-                                      stream=None):
+                                      stream=None, weight_kind: int = DVP_WEIGHT_NONE,
+                                      weight_lo: float = 0.0, weight_hi: float = 1.0):
     """Pruned log-probabilities and gradients with respect to ``hidden`` and
     ``w_vocab`` with the training logits hidden x w_vocab^T produced panel by
-    panel inside the library and never stored as a [T, V] matrix."""
+    panel inside the library and never stored as a [T, V] matrix.  With
+    ``weight_kind`` (truncate or mask, finite ``weight_hi``) each token's upstream
+    gradient is multiplied by its importance weight; the weights come back as
+    ``weight``."""
     lib = load_library()
     _check_matrix("hidden", hidden)
     _check_matrix("w_vocab", w_vocab)
@@ -452,6 +460,11 @@ def dvp_fused_lmhead_forward_backward(hidden: torch.Tensor, w_vocab: torch.Tenso
     res.workspace = workspace
     a.workspace, a.workspace_bytes = _ptr(workspace), workspace.numel() * workspace.element_size()
     a.stream = _stream(stream)
+    a.weight_kind = int(weight_kind)
+    if weight_kind != DVP_WEIGHT_NONE:
+        a.weight_lo, a.weight_hi = float(weight_lo), float(weight_hi)
+        res.weight = torch.empty(T, dtype=torch.float32, device=dev)
+        a.weight_out = _ptr(res.weight)
     st = lib.dvp_fused_lmhead_forward_backward(ctypes.byref(a))
     if st != DVP_OK:
         raise DvpError(st, "dvp_fused_lmhead_forward_backward")

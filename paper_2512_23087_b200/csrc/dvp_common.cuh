@@ -301,6 +301,10 @@ struct RowParams {
   int weight_kind;  // DVP_WEIGHT_*: the upstream gradient is multiplied by the token's importance weight
   float weight_lo, weight_hi;
   float *weight_out;
+  // the inference side of the weight when an earlier launch computed it (no `infer` matrix then):
+  // ln pi^mp_infer(a) per token, and flags whose DVP_FLAG_IN_TRAIN bit says "a in V'_S"
+  const float *given_logp_mp_i;
+  const uint8_t *given_flags_i;
 };
 
 __device__ __forceinline__ long long load_id(const void *ids, int is_i32, long long t) {
@@ -414,6 +418,15 @@ __device__ __forceinline__ float row_weight(const RowParams &p, const SideStats 
   const float lt = logp_mp_of(st), li = logp_mp_of(si);
   const float r = (p.mode & DVP_MODE_FINITE_MASK) ? lt - li : log_ratio_of(st.member, si.member, lt, li);
   return token_weight(r, p.weight_kind, p.weight_lo, p.weight_hi);
+}
+
+// The same from an inference side computed by an earlier launch.
+__device__ __forceinline__ float row_weight_given(const RowParams &p, const SideStats &st, long long t,
+                                                  bool valid_id) {
+  if (!valid_id) return __int_as_float(0x7fc00000);
+  const float lt = logp_mp_of(st), li = p.given_logp_mp_i[t];
+  const bool in_i = (p.given_flags_i[t] & DVP_FLAG_IN_TRAIN) != 0;
+  return token_weight(log_ratio_of(st.member, in_i, lt, li), p.weight_kind, p.weight_lo, p.weight_hi);
 }
 
 // Arguments of the stand-alone backward map.

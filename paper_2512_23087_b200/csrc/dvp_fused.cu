@@ -85,7 +85,8 @@ struct FusedScalars {
 };
 
 // scale = 2^(14 - x) with max|g| < 2^x, so that |scale * G| < 2^14.
-__global__ void grad_scale_kernel(const float *upstream, long long T, FusedScalars *out) {
+// `factor` bounds what the kernel multiplies into the upstream gradients (an importance weight).
+__global__ void grad_scale_kernel(const float *upstream, long long T, float factor, FusedScalars *out) {
   __shared__ float red[32];
   float m = 0.f;
   for (long long t = threadIdx.x; t < T; t += blockDim.x) {
@@ -97,6 +98,7 @@ __global__ void grad_scale_kernel(const float *upstream, long long T, FusedScala
   __syncthreads();
   if (threadIdx.x == 0) {
     for (int w = 1; w < (int)(blockDim.x >> 5); ++w) m = fmaxf(m, red[w]);
+    m *= factor;
     int x = 0;
     if (m > 0.f) frexpf(m, &x);
     int e = 14 - x;
@@ -222,6 +224,14 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
     return DVP_ERR_INVALID_ARG;
   if (a->infer_logits && a->ld_infer < a->V) return DVP_ERR_INVALID_ARG;
   if (!a->infer_logits && a->log_ratio) return DVP_ERR_INVALID_ARG;
+  if (a->weight_kind != DVP_WEIGHT_NONE) {
+    if (a->weight_kind != DVP_WEIGHT_TRUNCATE && a->weight_kind != DVP_WEIGHT_MASK) return DVP_ERR_INVALID_ARG;
+    if (!a->infer_logits) return DVP_ERR_INVALID_ARG;
+    if (!(a->weight_lo >= 0.f && a->weight_hi >= a->weight_lo) || !std::isfinite(a->weight_hi))
+      return DVP_ERR_INVALID_ARG;
+  } else if (a->weight_out) {
+    return DVP_ERR_INVALID_ARG;
+  }
   if (a->ld_hidden % 8 || a->ld_w % 8 || a->ld_dh % 8 || a->ld_dw % 8 ||
       (uintptr_t)a->hidden % 16 || (uintptr_t)a->w_vocab % 16 || (uintptr_t)a->d_hidden % 32 ||
       (uintptr_t)a->d_w % 32)
@@ -252,12 +262,30 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
   const long long id_bytes = a->id_dtype == DVP_ID_I32 ? 4 : 8;
   const long long mask_words = (a->V + 31) / 32;
 
-  grad_scale_kernel<<<1, 1024, 0, s>>>(a->upstream, a->T, sc);
+  const bool weighted = a->weight_kind != DVP_WEIGHT_NONE;
+  grad_scale_kernel<<<1, 1024, 0, s>>>(a->upstream, a->T, weighted ? fmaxf(1.f, a->weight_hi) : 1.f, sc);
   launch_transpose<__nv_bfloat16, __half>(w, a->ld_w, wt16, L.Vp, V, H, s);
   launch_transpose<__nv_bfloat16, __half>(hidden, a->ld_hidden, ht16, L.Tp, T, H, s);
   if (cudaGetLastError() != cudaSuccess) return DVP_ERR_CUDA;
 
   const double log_rho = a->rho > 0.0 ? std::log(a->rho) : -HUGE_VAL;
+  // the inference rows: an ordinary forward-only row pass over the stored logits
+  auto infer_rows = [&]() -> cudaError_t {
+    RowParams p{};
+    p.train = a->infer_logits;
+    p.ids = a->ids;
+    p.T = a->T;
+    p.V = a->V;
+    p.ld_train = a->ld_infer;
+    p.log_rho = log_rho;
+    p.id_is_i32 = a->id_dtype == DVP_ID_I32;
+    p.out_t = a->infer;
+    p.out_t.logp_mp = lpi;
+    p.flags = fli;
+    return launch_row_kernels(p, DVP_BF16, DVP_BF16, 0, s);
+  };
+  // with an importance weight the training rows need the inference side first
+  if (weighted && infer_rows() != cudaSuccess) return DVP_ERR_CUDA;
   int panel_index = 0;
   for (long long r0 = 0; r0 < a->T; r0 += L.panel, ++panel_index) {
     const int rows = (int)((a->T - r0 < L.panel) ? a->T - r0 : L.panel);
@@ -281,6 +309,14 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
     p.out_t = offset_side(a->train, r0, mask_words);
     p.out_t.logp_mp = lpt + r0;
     p.flags = flt + r0;
+    if (weighted) {
+      p.weight_kind = (int)a->weight_kind;
+      p.weight_lo = a->weight_lo;
+      p.weight_hi = a->weight_hi;
+      p.weight_out = a->weight_out ? a->weight_out + r0 : nullptr;
+      p.given_logp_mp_i = lpi + r0;
+      p.given_flags_i = fli + r0;
+    }
     if (launch_row_kernels(p, DVP_F32, DVP_F16, 0, s) != cudaSuccess) return DVP_ERR_CUDA;
     launch_transpose<__half, __half>(g16, L.Vp, gt16, L.panel, rows, V, s);
     // d_hidden[r0 : r0 + rows] = G x W / scale
@@ -295,18 +331,7 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
   }
 
   if (a->infer_logits) {
-    RowParams p{};
-    p.train = a->infer_logits;
-    p.ids = a->ids;
-    p.T = a->T;
-    p.V = a->V;
-    p.ld_train = a->ld_infer;
-    p.log_rho = log_rho;
-    p.id_is_i32 = a->id_dtype == DVP_ID_I32;
-    p.out_t = a->infer;
-    p.out_t.logp_mp = lpi;
-    p.flags = fli;
-    if (launch_row_kernels(p, DVP_BF16, DVP_BF16, 0, s) != cudaSuccess) return DVP_ERR_CUDA;
+    if (!weighted && infer_rows() != cudaSuccess) return DVP_ERR_CUDA;
     combine_sides_kernel<<<(unsigned)((a->T + 255) / 256), 256, 0, s>>>(a->T, lpt, lpi, fli, flt,
                                                                         a->log_ratio);
   }

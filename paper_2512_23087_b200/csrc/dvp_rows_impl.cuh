@@ -559,7 +559,7 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
   uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * ((p.V + 31) / 32) : nullptr;
   HotList hot;
   SideStats st, si;
-  if constexpr (kWeighted) {  // the launcher guarantees an inference matrix
+  if (kWeighted && p.infer) {  // otherwise an earlier launch left the inference side's results
     const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
     uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
     HotList hot_i;
@@ -573,7 +573,7 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
   if (p.grad) {
     float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
     if constexpr (kWeighted) {
-      const float w = row_weight(p, st, si, a >= 0);
+      const float w = p.infer ? row_weight(p, st, si, a >= 0) : row_weight_given(p, st, t, a >= 0);
       if (w == w) g *= w;
       if (p.weight_out && threadIdx.x == 0 && rank == 0) p.weight_out[t] = w;
     }
@@ -677,7 +677,8 @@ __global__ void dvp_row_kernel_scalar(const RowParams p) {
   SideStats si;
   if (irow) si = row_stats_scalar<TIn>(irow, p.V, a, p.log_rho, p.mode, p.mask_value, scratch, mask_i);
   float w = 1.f;
-  if (p.weight_kind != DVP_WEIGHT_NONE && irow) w = row_weight(p, st, si, a >= 0);
+  if (p.weight_kind != DVP_WEIGHT_NONE)
+    w = irow ? row_weight(p, st, si, a >= 0) : row_weight_given(p, st, t, a >= 0);
   if (p.weight_out && threadIdx.x == 0) p.weight_out[t] = w;
 
   if (p.grad) {
@@ -808,7 +809,7 @@ static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s
   int threads = hint & 0xffff, stage = (hint >> 16) & 0xff, cluster = (hint >> 24) & 0xff;
   // stage byte 0x11: the kernel that keeps the row in shared memory; 0x1e: the same with
   // block 0's first copy withheld (self-test of the wait limit)
-  if (stage == 0x11 || stage == 0x1e) {
+  if ((stage == 0x11 || stage == 0x1e) && !p.given_logp_mp_i) {
     const bool ok16 = aligned32(p.train, p.ld_train, sizeof(TIn)) &&
                       aligned32(p.infer, p.ld_infer, sizeof(TIn)) &&
                       aligned32(p.grad, p.ld_grad, sizeof(TGrad));

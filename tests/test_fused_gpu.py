@@ -68,7 +68,9 @@ def test_gemm_tn_padded_strides_and_argument_errors():
     assert e.value.status == binding.DVP_ERR_UNSUPPORTED
 
 
-def _check_fused(batch, rho, res, want, V):
+def _check_fused(batch, rho, res, want, V, weight=None):
+    """weight: (kind, lo, hi) of an importance-weighted call; rows whose ratio sits within 5e-4
+    relative of a masking bound (where the weight jumps) are left out of the gradient rows."""
     rep = {}
     z = want.logits
     H = batch.hidden.shape[1]
@@ -117,21 +119,35 @@ def _check_fused(batch, rho, res, want, V):
         assert (num <= bound).all(), f"{name}: worst {np.max(num / np.maximum(den, 1e-300)):.3e}"
         rep[name] = float(np.max(num / np.maximum(den, 1e-6 * den.max())))
 
+    if weight is not None:
+        ratio = np.exp(want.rows.log_ratio)
+        near = np.zeros(len(ratio), dtype=bool)
+        if weight[0] == oracle.WEIGHT_MASK:
+            with np.errstate(invalid="ignore"):
+                near = (np.abs(ratio - weight[1]) <= 5e-4 * weight[1]) | (np.abs(ratio - weight[2]) <= 5e-4 * weight[2])
+        rep["near_weight_bound_rows"] = int(near.sum())
+        ok = ok & ~near
+        got_w = res.weight.cpu().numpy().astype(np.float64)
+        assert np.array_equal(np.isnan(got_w), np.isnan(want.rows.weight))
+        assert (np.abs(got_w - want.rows.weight)[ok] <= 2e-4 * np.abs(want.rows.weight[ok]) + 1e-12).all(), "weight"
+        rep["zero_weight_rows"] = int((want.rows.weight[ok] == 0).sum())
     rows_close(res.d_hidden, want.d_hidden, "d_hidden", ok)
     if ok.all():
         rows_close(res.d_w, want.d_w, "d_w")
     return rep
 
 
-def _run_fused(T, H, V, rho, seed, **kw):
+def _run_fused(T, H, V, rho, seed, weight=None, **kw):
     w = inputs.WORKLOADS["c4_fused_lmhead"]
     batch = inputs.make_fused(w, seed=seed, device=DEV, T=T, H=H, V=V)
+    wkw = {} if weight is None else dict(weight_kind=weight[0], weight_lo=weight[1], weight_hi=weight[2])
     res = binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, rho,
-                                                    batch.upstream, infer_logits=batch.infer, **kw)
+                                                    batch.upstream, infer_logits=batch.infer, **wkw, **kw)
     torch.cuda.synchronize()
     assert res.workspace[:4].view(torch.int32).item() == 0, "a tensor-core kernel gave up waiting"
     want = oracle.dvp_fused_lmhead(_bits(batch.hidden), _bits(batch.w_vocab), _bits(batch.infer),
-                                   batch.ids.cpu().numpy(), rho, batch.upstream.cpu().numpy().astype(np.float64))
+                                   batch.ids.cpu().numpy(), rho, batch.upstream.cpu().numpy().astype(np.float64),
+                                   **wkw)
     return batch, res, want
 
 
@@ -140,6 +156,25 @@ def _run_fused(T, H, V, rho, seed, **kw):
 def test_fused_lmhead_small(T, H, V, rho):
     batch, res, want = _run_fused(T, H, V, rho, seed=T)
     _check_fused(batch, rho, res, want, V)
+
+
+@pytest.mark.parametrize("weight", [(oracle.WEIGHT_TRUNCATE, 0.0, 1.004), (oracle.WEIGHT_MASK, 0.985, 1.01)],
+                         ids=["truncate", "mask"])
+@pytest.mark.parametrize("T,H,V,rho,panel", [(200, 256, 3000, 1e-3, 0), (300, 128, 2048, 1e-2, 128)])
+def test_fused_lmhead_importance_weighted(T, H, V, rho, panel, weight):
+    """Thm. 5.3 per token through the LM head: the inference rows are swept first, the
+    training panels take the weight from them; one panel and several."""
+    batch, res, want = _run_fused(T, H, V, rho, seed=T + 1, weight=weight, panel_rows=panel)
+    rep = _check_fused(batch, rho, res, want, V, weight=weight)
+    assert (want.rows.weight != np.exp(want.rows.log_ratio))[np.isfinite(want.rows.log_ratio)].any()   # the bounds do cut
+    if weight[0] == oracle.WEIGHT_MASK:
+        assert rep["zero_weight_rows"] >= 1
+    plain = binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, rho, batch.upstream,
+                                                      infer_logits=batch.infer, panel_rows=panel)
+    torch.cuda.synchronize()
+    assert torch.equal(plain.train.logp_mp, res.train.logp_mp) and torch.equal(plain.flags, res.flags)
+    fin = torch.isfinite(plain.log_ratio)
+    assert torch.equal(plain.log_ratio[fin], res.log_ratio[fin])
 
 
 def test_fused_lmhead_several_panels_and_dw_accumulation():
