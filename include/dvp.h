@@ -407,7 +407,9 @@ int dvp_fused_lmhead_forward_backward_static(const dvp_fused_args *args);
  *   a, b, c   device; lda, ldb, ldc multiples of 8; a, b 16-byte, c 32-byte aligned
  *   accumulate  bit 0: add to C instead of overwriting it; bit 1: use the kernel that
  *             gives each 128 x 256 tile to one block instead of 256 x 256 tiles to
- *             pairs of blocks (same results up to summation order; for comparison)
+ *             pairs of blocks (same results up to summation order; for comparison);
+ *             bit 2: `a` points to A transposed, [k, m] with m contiguous and row
+ *             stride lda (not with bit 1): the tensor cores read it as it lies
  *   status    device int32, written non-zero if a kernel gave up waiting
  * Errors: DVP_ERR_INVALID_ARG (null pointers, negative sizes),
  * DVP_ERR_UNSUPPORTED (dtype, alignment), DVP_ERR_CUDA.

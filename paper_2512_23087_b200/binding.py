@@ -383,23 +383,26 @@ def dvp_row_wait_status() -> int:
 
 
 def dvp_gemm_tn(a: torch.Tensor, b: torch.Tensor, *, alpha: float = 1.0, out: torch.Tensor | None = None,
-                accumulate: bool = False, single_block_tiles: bool = False, stream=None):
+                accumulate: bool = False, single_block_tiles: bool = False, stream=None,
+                a_transposed: bool = False):
     """``out (+)= alpha * a @ b.T`` on the tensor cores; a [m, k] and b [n, k] are
-    both bf16 or both f16 with k contiguous, out is float32.  Returns (out, status)
-    where status is a device int32 that is non-zero if the kernel gave up waiting."""
+    both bf16 or both f16 with k contiguous, out is float32.  With ``a_transposed``
+    ``a`` is given as [k, m] with m contiguous (``out (+)= alpha * a.T @ b.T``).
+    Returns (out, status) where status is a device int32 that is non-zero if the
+    kernel gave up waiting."""
     lib = load_library()
     _check_matrix("a", a)
     _check_matrix("b", b)
     if a.dtype != b.dtype or a.dtype not in (torch.bfloat16, torch.float16):
         raise TypeError("a and b must both be bfloat16 or both float16")
-    m, k = a.shape
+    m, k = (a.shape[1], a.shape[0]) if a_transposed else a.shape
     n = b.shape[0]
     if out is None:
         out = torch.empty(m, n, dtype=torch.float32, device=a.device)
     status = torch.zeros(1, dtype=torch.int32, device=a.device)
+    mode = int(accumulate) | (2 if single_block_tiles else 0) | (4 if a_transposed else 0)
     st = lib.dvp_gemm_tn(_ptr(a), a.stride(0), _ptr(b), b.stride(0), _ptr(out), out.stride(0), m, n, k,
-                         _DTYPES[a.dtype], float(alpha), int(accumulate) | (2 if single_block_tiles else 0),
-                         _ptr(status), _stream(stream))
+                         _DTYPES[a.dtype], float(alpha), mode, _ptr(status), _stream(stream))
     if st != DVP_OK:
         raise DvpError(st, "dvp_gemm_tn")
     return out, status

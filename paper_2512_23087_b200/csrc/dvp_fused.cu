@@ -128,7 +128,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct FusedLayout {
   long long Vp, Tp, panel;
-  size_t off_scalars, off_lpt, off_lpi, off_fli, off_flt, off_wt, off_ht, off_z, off_g, off_gt, total;
+  size_t off_scalars, off_lpt, off_lpi, off_fli, off_flt, off_wt, off_ht, off_z, off_g, total;
 };
 
 bool fused_layout(const dvp_fused_args *a, FusedLayout *L) {
@@ -159,7 +159,6 @@ bool fused_layout(const dvp_fused_args *a, FusedLayout *L) {
   L->off_ht = take((size_t)a->H * L->Tp * 2);
   L->off_z = take((size_t)panel * L->Vp * 4);
   L->off_g = take((size_t)panel * L->Vp * 2);
-  L->off_gt = take((size_t)a->V * panel * 2);
   L->total = o;
   return true;
 }
@@ -203,7 +202,7 @@ int dvp_gemm_tn(const void *a, int64_t lda, const void *b, int64_t ldb, float *c
   const cudaError_t e =
       dvp::gemm::launch_gemm_tn(a, lda, b, ldb, c, ldc, (int)m, (int)n, (int)k, dtype == DVP_BF16, alpha,
                                 nullptr, (accumulate & 1) != 0, status, sms,
-                                static_cast<cudaStream_t>(stream), (accumulate & 2) != 0);
+                                static_cast<cudaStream_t>(stream), (accumulate & 2) != 0, (accumulate & 4) != 0);
   if (e == cudaErrorInvalidValue) return DVP_ERR_UNSUPPORTED;
   return e == cudaSuccess ? DVP_OK : DVP_ERR_CUDA;
 }
@@ -255,7 +254,6 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
   __half *ht16 = reinterpret_cast<__half *>(ws + L.off_ht);   // [H, Tp]: hidden^T
   float *z = reinterpret_cast<float *>(ws + L.off_z);         // [panel, Vp] logits
   __half *g16 = reinterpret_cast<__half *>(ws + L.off_g);     // [panel, Vp] scaled gradient
-  __half *gt16 = reinterpret_cast<__half *>(ws + L.off_gt);   // [V, panel]: its transpose
   const __nv_bfloat16 *hidden = static_cast<const __nv_bfloat16 *>(a->hidden);
   const __nv_bfloat16 *w = static_cast<const __nv_bfloat16 *>(a->w_vocab);
   const int T = (int)a->T, H = (int)a->H, V = (int)a->V;
@@ -318,15 +316,15 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
       p.given_flags_i = fli + r0;
     }
     if (launch_row_kernels(p, DVP_F32, DVP_F16, 0, s) != cudaSuccess) return DVP_ERR_CUDA;
-    launch_transpose<__half, __half>(g16, L.Vp, gt16, L.panel, rows, V, s);
     // d_hidden[r0 : r0 + rows] = G x W / scale
     e = gemm::launch_gemm_tn(g16, L.Vp, wt16, L.Vp, a->d_hidden + r0 * a->ld_dh, a->ld_dh, rows, H, V,
                              false, 1.f, &sc->inv_scale, false, &sc->status, sms, s);
     if (e != cudaSuccess) return e == cudaErrorInvalidValue ? DVP_ERR_UNSUPPORTED : DVP_ERR_CUDA;
-    // d_w (+)= G^T x hidden[r0 : r0 + rows] / scale
-    e = gemm::launch_gemm_tn(gt16, L.panel, ht16 + r0, L.Tp, a->d_w, a->ld_dw, V, H, rows, false, 1.f,
+    // d_w (+)= G^T x hidden[r0 : r0 + rows] / scale: G is read as it lies, [rows, V] with V
+    // contiguous, as the transposed (MN-major) A operand of the contraction
+    e = gemm::launch_gemm_tn(g16, L.Vp, ht16 + r0, L.Tp, a->d_w, a->ld_dw, V, H, rows, false, 1.f,
                              &sc->inv_scale, panel_index > 0 || a->accumulate_dw != 0, &sc->status, sms,
-                             s);
+                             s, false, true);
     if (e != cudaSuccess) return e == cudaErrorInvalidValue ? DVP_ERR_UNSUPPORTED : DVP_ERR_CUDA;
   }
 

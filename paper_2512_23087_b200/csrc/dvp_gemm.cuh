@@ -43,6 +43,7 @@ struct Params {
   const float *alpha_dev;  // optional device scalar multiplied into alpha
   int accumulate;          // C += instead of C =
   int *status;             // device word, set non-zero when a wait gives up
+  int a_mn_major;          // A is stored transposed, [K, M] with M contiguous (pair kernel only)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -98,6 +99,20 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
   d |= (uint64_t)(1024 >> 4) << 32;         // stride byte offset between 8-row groups
   d |= (uint64_t)1 << 46;                   // descriptor version of this architecture
   d |= (uint64_t)2 << 61;                   // 128-byte swizzle
+  return d;
+}
+
+// The same for an MN-major operand (stored [K, MN] with MN contiguous), brought in as
+// boxes of 64 K-rows x 64 MN-elements: inside a box a K-row is 128 swizzled bytes, groups
+// of 8 K-rows are 1024 bytes apart (stride byte offset), and the next 64 MN-elements
+// start one box (8192 bytes) further (leading byte offset).
+__device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+  d |= (uint64_t)(8192 >> 4) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
   return d;
 }
 
@@ -446,7 +461,13 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           if (rank == 0) mbar_expect_tx(bar_local, 2 * kStageBytes2);
           const uint32_t bar = map_to_rank(bar_local, 0);
           const uint32_t dst = base + s * kStageBytes2;
-          tma_load_2d_pair(dst, &map_a, bar, ks * kBK, tm * kPairBM + (int)rank * kBM);
+          if (p.a_mn_major) {  // two boxes of 64 K-rows x 64 rows of A
+            const int m0 = tm * kPairBM + (int)rank * kBM;
+            tma_load_2d_pair(dst, &map_a, bar, m0, ks * kBK);
+            tma_load_2d_pair(dst + kBytesA / 2, &map_a, bar, m0 + 64, ks * kBK);
+          } else {
+            tma_load_2d_pair(dst, &map_a, bar, ks * kBK, tm * kPairBM + (int)rank * kBM);
+          }
           tma_load_2d_pair(dst + kBytesA, &map_b, bar, ks * kBK, tn * kBN + (int)rank * (kBN / 2));
         }
       }
@@ -455,7 +476,9 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ---------------- MMA issuer (leader block only)
     if (lane == 0 && rank == 0) {
       const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kBN >> 3) << 17) |
-                             ((uint32_t)(kPairBM >> 4) << 24);
+                             ((uint32_t)(kPairBM >> 4) << 24) | (p.a_mn_major ? (1u << 15) : 0u);
+      // bytes between two K = 16 steps of A: 32 inside a K-major row, 16 K-rows of an MN-major box
+      const uint32_t a_step_bytes = p.a_mn_major ? 16u * 128u : (uint32_t)(kUmmaK * 2);
       uint32_t it = 0, local_tile = 0;
       for (int tile = pair; tile < n_tiles && !*abort_flag; tile += n_pairs, ++local_tile) {
         const uint32_t buf = local_tile & 1, use = local_tile >> 1;
@@ -475,11 +498,13 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           }
           tc_fence_after();
           const uint32_t a_addr = base + s * kStageBytes2, b_addr = a_addr + kBytesA;
-          const uint64_t adesc = smem_desc_sw128(a_addr), bdesc = smem_desc_sw128(b_addr);
+          const uint64_t adesc = p.a_mn_major ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
+          const uint64_t bdesc = smem_desc_sw128(b_addr);
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             const uint64_t step = (uint64_t)((k * kUmmaK * 2) >> 4);
-            umma_pair(tmem_d, adesc + step, bdesc + step, idesc, (ks > 0 || k > 0) ? 1u : 0u);
+            const uint64_t a_step = (uint64_t)((k * a_step_bytes) >> 4);
+            umma_pair(tmem_d, adesc + a_step, bdesc + step, idesc, (ks > 0 || k > 0) ? 1u : 0u);
           }
           umma_commit_pair(smem_u32(&sh->empty[s]));
         }
@@ -600,16 +625,19 @@ inline bool make_map(CUtensorMap *map, const void *base, long long rows, long lo
 inline cudaError_t launch_gemm_tn(const void *A, long long lda, const void *B, long long ldb, float *C,
                                   long long ldc, int M, int N, int K, bool is_bf16, float alpha,
                                   const float *alpha_dev, bool accumulate, int *status, int sm_count,
-                                  cudaStream_t stream, bool single_block_tiles = false) {
+                                  cudaStream_t stream, bool single_block_tiles = false,
+                                  bool a_mn_major = false) {
   if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
   if (lda % 8 || ldb % 8 || ldc % 8 || (uintptr_t)A % 16 || (uintptr_t)B % 16 || (uintptr_t)C % 32)
     return cudaErrorInvalidValue;
-  Params p{C, ldc, M, N, K, alpha, alpha_dev, accumulate ? 1 : 0, status};
+  if (a_mn_major && single_block_tiles) return cudaErrorInvalidValue;
+  Params p{C, ldc, M, N, K, alpha, alpha_dev, accumulate ? 1 : 0, status, a_mn_major ? 1 : 0};
   CUtensorMap map_a, map_b;
   if (!single_block_tiles) {
-    // pairs of blocks on 256 x 256 tiles
-    if (!make_map(&map_a, A, M, K, lda, kBM, is_bf16) || !make_map(&map_b, B, N, K, ldb, kBN / 2, is_bf16))
-      return cudaErrorInvalidValue;
+    // pairs of blocks on 256 x 256 tiles; a transposed A is [K, M]: its "rows" are K, boxes of 64 x 64
+    const bool ok_a = a_mn_major ? make_map(&map_a, A, K, M, lda, 64, is_bf16)
+                                 : make_map(&map_a, A, M, K, lda, kBM, is_bf16);
+    if (!ok_a || !make_map(&map_b, B, N, K, ldb, kBN / 2, is_bf16)) return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(gemm_tn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)kSmemBytes2);
     if (e != cudaSuccess) return e;

@@ -54,6 +54,31 @@ def test_gemm_tn_matches_float64_matmul(dtype, m, n, k, single):
     assert (out2.double() - 0.75 * ref).abs().max().item() <= 2 * tol
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("m,n,k", [(256, 256, 64), (512, 256, 256), (304, 520, 200), (8, 8, 8), (1000, 776, 1032),
+                                   (4104, 512, 4096), (2048, 264, 8200)])
+def test_gemm_tn_transposed_a_operand(dtype, m, n, k):
+    """A given as [k, m] with m contiguous: the tensor cores read it as an MN-major
+    operand (this is how d_w = G^T hidden takes the gradient panel without a transpose)."""
+    g = torch.Generator(device=DEV).manual_seed(m * 5 + n * 3 + k)
+    at = torch.randn(k, m + 8, generator=g, device=DEV).to(dtype)[:, :m]      # padded row stride
+    b = torch.randn(n, k, generator=g, device=DEV).to(dtype)
+    ref = at.double().t() @ b.double().t()
+    out, status = binding.dvp_gemm_tn(at, b, alpha=0.5, a_transposed=True)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    tol = (2.0 ** -24 * (k / 16) + 1e-6) * ref.abs().max().item()
+    assert (out.double() - 0.5 * ref).abs().max().item() <= tol
+    plain, _ = binding.dvp_gemm_tn(at.t().contiguous(), b, alpha=0.5)
+    torch.cuda.synchronize()
+    assert (out - plain).abs().max().item() <= 2 * tol
+    out2, status = binding.dvp_gemm_tn(at, b, alpha=0.25, out=out.clone(), accumulate=True, a_transposed=True)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and (out2.double() - 0.75 * ref).abs().max().item() <= 2 * tol
+    with pytest.raises(binding.DvpError):          # only the paired kernel reads a transposed A
+        binding.dvp_gemm_tn(at, b, a_transposed=True, single_block_tiles=True)
+
+
 def test_gemm_tn_padded_strides_and_argument_errors():
     g = torch.Generator(device=DEV).manual_seed(5)
     a = torch.randn(200, 328, generator=g, device=DEV).to(torch.bfloat16)[:, :320]
