@@ -378,7 +378,7 @@ int dvp_monitor(const dvp_monitor_args *args);
  * nothing, on the device or through any library.
  *
  * Limit: the workspace the arguments need (dvp_workspace_bytes with the same
- * panel_rows; roughly (2 H + 8 panel_rows) V + 2 H T bytes) must fit in
+ * panel_rows; roughly (2 H + 6 panel_rows) V + 2 H T bytes) must fit in
  * DVP_STATIC_WORKSPACE_BYTES, e.g. H = 1024, V = 8192, any T up to a few
  * thousand.  Larger problems return DVP_ERR_WORKSPACE and launch nothing.
  * Other errors are those of dvp_fused_lmhead_forward_backward;
