@@ -409,7 +409,10 @@ int dvp_fused_lmhead_forward_backward_static(const dvp_fused_args *args);
  *             gives each 128 x 256 tile to one block instead of 256 x 256 tiles to
  *             pairs of blocks (same results up to summation order; for comparison);
  *             bit 2: `a` points to A transposed, [k, m] with m contiguous and row
- *             stride lda (not with bit 1): the tensor cores read it as it lies
+ *             stride lda (not with bit 1): the tensor cores read it as it lies;
+ *             bit 3: every output tile is computed as two halves of the k range
+ *             that are added into C with atomics (for few tiles and a long k;
+ *             with two addends the sum does not depend on their order)
  *   status    device int32, written non-zero if a kernel gave up waiting
  * Errors: DVP_ERR_INVALID_ARG (null pointers, negative sizes),
  * DVP_ERR_UNSUPPORTED (dtype, alignment), DVP_ERR_CUDA.

@@ -384,10 +384,11 @@ def dvp_row_wait_status() -> int:
 
 def dvp_gemm_tn(a: torch.Tensor, b: torch.Tensor, *, alpha: float = 1.0, out: torch.Tensor | None = None,
                 accumulate: bool = False, single_block_tiles: bool = False, stream=None,
-                a_transposed: bool = False):
+                a_transposed: bool = False, split_k: bool = False):
     """``out (+)= alpha * a @ b.T`` on the tensor cores; a [m, k] and b [n, k] are
     both bf16 or both f16 with k contiguous, out is float32.  With ``a_transposed``
     ``a`` is given as [k, m] with m contiguous (``out (+)= alpha * a.T @ b.T``).
+    ``split_k`` computes every tile as two halves of the k range added into ``out``.
     Returns (out, status) where status is a device int32 that is non-zero if the
     kernel gave up waiting."""
     lib = load_library()
@@ -400,7 +401,7 @@ def dvp_gemm_tn(a: torch.Tensor, b: torch.Tensor, *, alpha: float = 1.0, out: to
     if out is None:
         out = torch.empty(m, n, dtype=torch.float32, device=a.device)
     status = torch.zeros(1, dtype=torch.int32, device=a.device)
-    mode = int(accumulate) | (2 if single_block_tiles else 0) | (4 if a_transposed else 0)
+    mode = int(accumulate) | (2 if single_block_tiles else 0) | (4 if a_transposed else 0) | (8 if split_k else 0)
     st = lib.dvp_gemm_tn(_ptr(a), a.stride(0), _ptr(b), b.stride(0), _ptr(out), out.stride(0), m, n, k,
                          _DTYPES[a.dtype], float(alpha), mode, _ptr(status), _stream(stream))
     if st != DVP_OK:

@@ -202,7 +202,8 @@ int dvp_gemm_tn(const void *a, int64_t lda, const void *b, int64_t ldb, float *c
   const cudaError_t e =
       dvp::gemm::launch_gemm_tn(a, lda, b, ldb, c, ldc, (int)m, (int)n, (int)k, dtype == DVP_BF16, alpha,
                                 nullptr, (accumulate & 1) != 0, status, sms,
-                                static_cast<cudaStream_t>(stream), (accumulate & 2) != 0, (accumulate & 4) != 0);
+                                static_cast<cudaStream_t>(stream), (accumulate & 2) != 0, (accumulate & 4) != 0,
+                                (accumulate & 8) ? 2 : 1);
   if (e == cudaErrorInvalidValue) return DVP_ERR_UNSUPPORTED;
   return e == cudaSuccess ? DVP_OK : DVP_ERR_CUDA;
 }
@@ -317,8 +318,11 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
     }
     if (launch_row_kernels(p, DVP_F32, DVP_F16, 0, s) != cudaSuccess) return DVP_ERR_CUDA;
     // d_hidden[r0 : r0 + rows] = G x W / scale
+    // few output tiles and a long K: two K ranges per tile fill the last wave of block pairs
+    const long long dh_tiles = ((rows + 255) / 256) * (long long)((H + 255) / 256);
     e = gemm::launch_gemm_tn(g16, L.Vp, wt16, L.Vp, a->d_hidden + r0 * a->ld_dh, a->ld_dh, rows, H, V,
-                             false, 1.f, &sc->inv_scale, false, &sc->status, sms, s);
+                             false, 1.f, &sc->inv_scale, false, &sc->status, sms, s, false, false,
+                             dh_tiles < 8LL * (sms / 2) ? 2 : 1);
     if (e != cudaSuccess) return e == cudaErrorInvalidValue ? DVP_ERR_UNSUPPORTED : DVP_ERR_CUDA;
     // d_w (+)= G^T x hidden[r0 : r0 + rows] / scale: G is read as it lies, [rows, V] with V
     // contiguous, as the transposed (MN-major) A operand of the contraction

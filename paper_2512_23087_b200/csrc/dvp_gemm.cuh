@@ -44,6 +44,8 @@ struct Params {
   int accumulate;          // C += instead of C =
   int *status;             // device word, set non-zero when a wait gives up
   int a_mn_major;          // A is stored transposed, [K, M] with M contiguous (pair kernel only)
+  int split_k;             // pair kernel: each tile's K range is cut into this many units whose
+                           // results are added to C with atomics (C zeroed or accumulated into)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -418,6 +420,9 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   const int n_tiles = tiles_m * tiles_n;
   const int k_slices = (p.K + kBK - 1) / kBK;
   const bool m_fastest = tiles_m <= tiles_n;
+  // work units: every tile once per K range; unit u is tile u % n_tiles of range u / n_tiles
+  const int n_units = n_tiles * p.split_k;
+  const int k_per = (k_slices + p.split_k - 1) / p.split_k;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages2; ++s) {
@@ -448,10 +453,12 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ---------------- producer (both blocks): own rows of A, own half of B
     if (lane == 0) {
       uint32_t it = 0;
-      for (int tile = pair; tile < n_tiles && !*abort_flag; tile += n_pairs) {
+      for (int unit = pair; unit < n_units && !*abort_flag; unit += n_pairs) {
+        const int tile = unit % n_tiles, k_lo = (unit / n_tiles) * k_per;
+        const int k_hi = min(k_slices, k_lo + k_per);
         const int tm = m_fastest ? tile % tiles_m : tile / tiles_n;
         const int tn = m_fastest ? tile / tiles_m : tile % tiles_n;
-        for (int ks = 0; ks < k_slices; ++ks, ++it) {
+        for (int ks = k_lo; ks < k_hi; ++ks, ++it) {
           const uint32_t s = it % kStages2, round = it / kStages2;
           if (round > 0 && !mbar_wait(smem_u32(&sh->empty[s]), (round - 1) & 1, abort_flag)) {
             if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, kErrProducerWait); }
@@ -480,7 +487,8 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       // bytes between two K = 16 steps of A: 32 inside a K-major row, 16 K-rows of an MN-major box
       const uint32_t a_step_bytes = p.a_mn_major ? 16u * 128u : (uint32_t)(kUmmaK * 2);
       uint32_t it = 0, local_tile = 0;
-      for (int tile = pair; tile < n_tiles && !*abort_flag; tile += n_pairs, ++local_tile) {
+      for (int unit = pair; unit < n_units && !*abort_flag; unit += n_pairs, ++local_tile) {
+        const int k_lo = (unit / n_tiles) * k_per, k_hi = min(k_slices, k_lo + k_per);
         const uint32_t buf = local_tile & 1, use = local_tile >> 1;
         if (use > 0 && !mbar_wait(smem_u32(&sh->tmem_empty[buf]), (use - 1) & 1, abort_flag)) {
           if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, kErrMmaWaitTmem); }
@@ -489,7 +497,7 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + buf * kBN;
         bool ok = true;
-        for (int ks = 0; ks < k_slices; ++ks, ++it) {
+        for (int ks = k_lo; ks < k_hi; ++ks, ++it) {
           const uint32_t s = it % kStages2, round = it / kStages2;
           if (!mbar_wait(smem_u32(&sh->full[s]), round & 1, abort_flag)) {
             if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, kErrMmaWaitFull); }
@@ -504,7 +512,7 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             const uint64_t step = (uint64_t)((k * kUmmaK * 2) >> 4);
             const uint64_t a_step = (uint64_t)((k * a_step_bytes) >> 4);
-            umma_pair(tmem_d, adesc + a_step, bdesc + step, idesc, (ks > 0 || k > 0) ? 1u : 0u);
+            umma_pair(tmem_d, adesc + a_step, bdesc + step, idesc, (ks > k_lo || k > 0) ? 1u : 0u);
           }
           umma_commit_pair(smem_u32(&sh->empty[s]));
         }
@@ -517,7 +525,8 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int quarter = warp & 3;
     const float alpha = p.alpha * (p.alpha_dev ? *p.alpha_dev : 1.f);
     uint32_t local_tile = 0;
-    for (int tile = pair; tile < n_tiles && !*abort_flag; tile += n_pairs, ++local_tile) {
+    for (int unit = pair; unit < n_units && !*abort_flag; unit += n_pairs, ++local_tile) {
+      const int tile = unit % n_tiles;
       const int tm = m_fastest ? tile % tiles_m : tile / tiles_n;
       const int tn = m_fastest ? tile / tiles_m : tile % tiles_n;
       const uint32_t buf = local_tile & 1, use = local_tile >> 1;
@@ -535,7 +544,9 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         tmem_wait_ld();
         const int col = tn * kBN + c0;
         if (row < p.M && col < p.N) {
-          if (col + 32 <= p.N) {
+          if (p.split_k > 1) {  // this unit holds a part of the sum: add it
+            for (int j = 0; j < 32 && col + j < p.N; ++j) atomicAdd(crow + col + j, alpha * __uint_as_float(r[j]));
+          } else if (col + 32 <= p.N) {
 #pragma unroll
             for (int j = 0; j < 32; j += 8) {
               uint32_t w[8];
@@ -626,12 +637,18 @@ inline cudaError_t launch_gemm_tn(const void *A, long long lda, const void *B, l
                                   long long ldc, int M, int N, int K, bool is_bf16, float alpha,
                                   const float *alpha_dev, bool accumulate, int *status, int sm_count,
                                   cudaStream_t stream, bool single_block_tiles = false,
-                                  bool a_mn_major = false) {
+                                  bool a_mn_major = false, int split_k = 1) {
   if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
   if (lda % 8 || ldb % 8 || ldc % 8 || (uintptr_t)A % 16 || (uintptr_t)B % 16 || (uintptr_t)C % 32)
     return cudaErrorInvalidValue;
   if (a_mn_major && single_block_tiles) return cudaErrorInvalidValue;
-  Params p{C, ldc, M, N, K, alpha, alpha_dev, accumulate ? 1 : 0, status, a_mn_major ? 1 : 0};
+  // every K range of a split needs work; the split results meet in C by atomic adds
+  if (single_block_tiles || split_k < 1 || (K + kBK - 1) / kBK < 2 * split_k) split_k = 1;
+  Params p{C, ldc, M, N, K, alpha, alpha_dev, accumulate ? 1 : 0, status, a_mn_major ? 1 : 0, split_k};
+  if (split_k > 1 && !accumulate) {
+    const cudaError_t z = cudaMemset2DAsync(C, (size_t)ldc * 4, 0, (size_t)N * 4, (size_t)M, stream);
+    if (z != cudaSuccess) return z;
+  }
   CUtensorMap map_a, map_b;
   if (!single_block_tiles) {
     // pairs of blocks on 256 x 256 tiles; a transposed A is [K, M]: its "rows" are K, boxes of 64 x 64
@@ -641,7 +658,7 @@ inline cudaError_t launch_gemm_tn(const void *A, long long lda, const void *B, l
     cudaError_t e = cudaFuncSetAttribute(gemm_tn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)kSmemBytes2);
     if (e != cudaSuccess) return e;
-    const int tiles = ((M + kPairBM - 1) / kPairBM) * ((N + kBN - 1) / kBN);
+    const int tiles = ((M + kPairBM - 1) / kPairBM) * ((N + kBN - 1) / kBN) * split_k;
     int pairs = sm_count / 2;
     if (pairs > tiles) pairs = tiles;
     cudaLaunchConfig_t cfg = {};

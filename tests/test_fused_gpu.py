@@ -79,6 +79,29 @@ def test_gemm_tn_transposed_a_operand(dtype, m, n, k):
         binding.dvp_gemm_tn(at, b, a_transposed=True, single_block_tiles=True)
 
 
+@pytest.mark.parametrize("m,n,k,transposed", [(256, 256, 8192, False), (1000, 776, 4104, False), (512, 264, 20000, True),
+                                              (300, 520, 200, False), (128, 256, 64, False)])
+def test_gemm_tn_split_k(m, n, k, transposed):
+    """Two halves of the k range per tile, met in C by atomic adds: same result as one
+    pass (up to the order of two partial sums), reruns bit-identical, accumulate on top."""
+    g = torch.Generator(device=DEV).manual_seed(m + n + k)
+    a = torch.randn(m, k, generator=g, device=DEV).to(torch.float16)
+    b = torch.randn(n, k, generator=g, device=DEV).to(torch.float16)
+    ref = a.double() @ b.double().t()
+    arg = a.t().contiguous() if transposed else a
+    out, status = binding.dvp_gemm_tn(arg, b, alpha=0.5, split_k=True, a_transposed=transposed)
+    out_b, _ = binding.dvp_gemm_tn(arg, b, alpha=0.5, split_k=True, a_transposed=transposed)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    tol = (2.0 ** -24 * (k / 16) + 1e-6) * ref.abs().max().item()
+    assert (out.double() - 0.5 * ref).abs().max().item() <= tol
+    assert torch.equal(out, out_b)
+    out2, status = binding.dvp_gemm_tn(arg, b, alpha=0.25, out=out.clone(), accumulate=True, split_k=True,
+                                       a_transposed=transposed)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and (out2.double() - 0.75 * ref).abs().max().item() <= 2 * tol
+
+
 def test_gemm_tn_padded_strides_and_argument_errors():
     g = torch.Generator(device=DEV).manual_seed(5)
     a = torch.randn(200, 328, generator=g, device=DEV).to(torch.bfloat16)[:, :320]
