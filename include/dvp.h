@@ -140,17 +140,24 @@ typedef struct {
  *   weight_out    device [T] float32 or NULL: the weight each token used (NaN
  *                 for a row without a valid sampled id)
  *   launch_hint   0 = library default; otherwise threads per block (a multiple
- *                 of 32, at most 512) in the low 16 bits, 0 or 2 in the next 8
- *                 bits, and the number of blocks that share one row (0, 1, 2 or
- *                 4; a thread-block cluster) in the top 8 bits.  0x11 in the
- *                 second byte (with zero elsewhere) selects the kernel that keeps
- *                 the row in shared memory (rows of up to 480 KB whose byte
- *                 length is a multiple of 16; others take the default kernel).
- *                 Tuning only: the safe set and counts do not depend on it.
- *                 0x1e there is a self-test of that kernel's wait limit: its
- *                 first block withholds its first copy, the wait for it runs out
- *                 after about a second, the launch ends by itself with undefined
- *                 outputs and dvp_row_wait_status reports code 1 or 2
+ *                 of 32, at most 512) in the low 16 bits, a kernel choice in the
+ *                 next 8 bits, and the number of blocks that share one row (0, 1, 2
+ *                 or 4; a thread-block cluster) in the top 8 bits.  Kernel choice:
+ *                 0 or 2 the default kernel (one sweep, then revisits of the 32-byte
+ *                 pieces of the row that can hold safe tokens); 3 or 4 (2-byte
+ *                 logits, at most 256 threads, no cluster) the kernel that keeps
+ *                 the candidates of the safe set in shared memory while the row
+ *                 streams and reads nothing twice, with 3 or 4 blocks per SM;
+ *                 0x11 (with zero elsewhere) the kernel that keeps the row itself
+ *                 in shared memory (rows of up to 480 KB whose byte length is a
+ *                 multiple of 16).  Rows a chosen kernel cannot take run the
+ *                 default one.  Tuning only: the safe set and counts do not
+ *                 depend on it.
+ *                 TEST ONLY: 0x1e in the second byte is a self-test of the 0x11
+ *                 kernel's wait limit, not an operating mode: its first block
+ *                 withholds its first copy, the wait for it runs out after about
+ *                 a second, the launch ends by itself with undefined outputs and
+ *                 dvp_row_wait_status reports code 1 or 2
  *
  * Rows whose start is 32-byte aligned in all three matrices take the
  * vectorised kernels; any other layout takes a scalar kernel, same results.

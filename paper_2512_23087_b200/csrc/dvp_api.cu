@@ -12,7 +12,7 @@ bool hint_ok(uint32_t hint) {
   if (threads != 0 && (threads % 32 != 0 || threads > 512)) return false;
   const uint32_t cluster = (hint >> 24) & 0xff;
   if (stage == 0x11 || stage == 0x1e) return cluster == 0;  // the resident-row kernel (0x1e: its self-test)
-  return (stage == 0 || stage == 2) && (cluster == 0 || cluster == 1 || cluster == 2 || cluster == 4);
+  return (stage == 0 || stage == 2 || stage == 3 || stage == 4) && (cluster == 0 || cluster == 1 || cluster == 2 || cluster == 4);
 }
 
 bool mode_ok(uint32_t mode, float mask_value) {

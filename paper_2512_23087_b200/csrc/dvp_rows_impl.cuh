@@ -768,6 +768,7 @@ __global__ void dvp_backward_kernel(const BackwardParams p) {
 
 }  // namespace dvp
 #include "dvp_rows_resident.cuh"
+#include "dvp_rows_store.cuh"
 namespace dvp {
 
 // ---- host-side launchers, instantiated once per logits type -------------------
@@ -803,10 +804,41 @@ static cudaError_t launch_rows_vec(const RowParams &p, int threads, size_t smem,
   }
 }
 
+// Shared memory one SM can give to `blocks` resident blocks (228 KB per SM, 1 KB of it
+// reserved per block), and the most one block may ask for.
+static inline size_t smem_per_block(int blocks) {
+  const size_t share = (size_t)228 * 1024 / blocks - 1024;
+  return share < (size_t)227 * 1024 ? share : (size_t)227 * 1024;
+}
+
+// The kernel that keeps the candidates of the safe set on chip (2-byte logits).
+template <typename TIn, typename TGrad, int kThreads, int kBlocks, bool kWeighted>
+static cudaError_t launch_rows_cs(const RowParams &p, int threads, int n_steps, cudaStream_t s) {
+  auto k = cs::dvp_row_kernel_cs<TIn, TGrad, kThreads, kBlocks, kWeighted>;
+  if (n_steps > 64) return cudaErrorNotSupported;  // positions are 16 bits
+  // as many list entries per warp as the SM's shared memory allows with kBlocks blocks
+  // resident, at most every element the warp sees
+  const size_t fixed = cs::smem_bytes_cs(threads, 0);
+  const size_t budget = smem_per_block(kBlocks * (kThreads / threads));
+  const int nwarp = threads / 32;
+  long long cap = budget > fixed ? (long long)((budget - fixed) / (4 * (size_t)nwarp)) : 0;
+  const long long most = (long long)n_steps * 64 * Granule<TIn>::kElems;
+  if (cap > most) cap = most;
+  if (cap < 32 * Granule<TIn>::kElems) return cudaErrorNotSupported;
+  const size_t smem = cs::smem_bytes_cs(threads, (int)cap);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  k<<<(unsigned)p.T, threads, smem, s>>>(p, n_steps, (int)cap);
+  return cudaGetLastError();
+}
+
 template <typename TIn, typename TGrad>
 static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s) {
   constexpr int kElems = Granule<TIn>::kElems;
   int threads = hint & 0xffff, stage = (hint >> 16) & 0xff, cluster = (hint >> 24) & 0xff;
+  const int stage_hint = stage;
   // stage byte 0x11: the kernel that keeps the row in shared memory; 0x1e: the same with
   // block 0's first copy withheld (self-test of the wait limit)
   if ((stage == 0x11 || stage == 0x1e) && !p.given_logp_mp_i) {
@@ -836,7 +868,26 @@ static cudaError_t launch_rows(const RowParams &p, uint32_t hint, cudaStream_t s
   const long long per = (long long)stage * threads;
   const size_t smem = (size_t)smem_words_fixed(threads) * 4 +
                       (size_t)((n_gran + per - 1) / per) * per * sizeof(uint16_t);
-  if (vec_ok && smem <= 200 * 1024) {
+  // 16-bit hot-list entries hold slot * 32 + lane: very long rows swept by few threads
+  // would not fit them
+  const bool hot_ok = ((n_gran + per - 1) / per) * stage * 32 <= 65536;
+  if constexpr (sizeof(TIn) == 2) {
+    // stage byte 3 or 4: the kernel that keeps the candidates of the safe set on chip, with
+    // three or four resident blocks per SM (measured slower than the kernel below; kept for
+    // comparison)
+    if (vec_ok && cluster == 1 && (stage_hint == 3 || stage_hint == 4) && threads <= 256) {
+      const int n_steps = (int)((n_gran + per - 1) / per);
+      cudaError_t e;
+      if (weighted)
+        e = launch_rows_cs<TIn, TGrad, 256, 3, true>(p, threads, n_steps, s);
+      else if (stage_hint == 3)
+        e = launch_rows_cs<TIn, TGrad, 256, 3, false>(p, threads, n_steps, s);
+      else
+        e = launch_rows_cs<TIn, TGrad, 256, 4, false>(p, threads, n_steps, s);
+      if (e != cudaErrorNotSupported) return e;
+    }
+  }
+  if (vec_ok && hot_ok && smem <= 200 * 1024) {
     if (cluster == 4 && threads <= 256 && stage == 2)
       return launch_rows_vec<TIn, TGrad, 2, 256, 4, 4>(p, threads, smem, s);
     if (cluster == 2 && threads <= 256 && stage == 2)
