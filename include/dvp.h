@@ -115,6 +115,13 @@ typedef struct {
   int32_t *count;   /* |V_S|                                                  */
   uint32_t *mask;   /* [T, ceil(V/32)] packed: bit (k%32) of word k/32 set    */
                     /* when k in V_S; padding bits of the last word are zero  */
+  float *log_cov;   /* ln Z, Z = sum_{k in V_S} pi(k) the coverage of Def. 5.2 */
+                    /* (<= 0; 1 - Z is the total variation distance between    */
+                    /* pi^mp and pi in the proof of Prop. 5.5).  Formed in     */
+                    /* double from the two sums the kernel holds, not from the */
+                    /* float outputs lse_safe and lse; Z itself is good to a    */
+                    /* few 1e-6, so 1 - Z keeps 1e-3 relative accuracy down to  */
+                    /* about 1 - Z = 4e-3                                      */
 } dvp_side_out;
 
 /*
@@ -316,9 +323,19 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *args);
  *   n_valid        device [S] int32: tokens with a sampled id
  *   n_zero_weight  device [S] int32: tokens with weight zero
  *   veto           device [S] bytes: 1 when some token weight < veto_threshold
+ *   log_cov        device [T] float32 or NULL: ln Z per token as written by
+ *                  dvp_forward (dvp_side_out.log_cov of the training side)
+ *   min_cov        device [S]: min over the sequence's tokens of the coverage Z
+ *                  (the Z_min of the bias bound of Prop. 5.5,
+ *                  |J_mp - J| <= R_max T (1 - Z_min)); +inf for an empty sequence
+ *   mean_cov       device [S]: mean of Z over the sequence's tokens (NaN if empty)
+ *                  min_cov and mean_cov need log_cov; every token counts, with
+ *                  or without a sampled id.  One sequence spanning [0, T) gives
+ *                  the batch-level figures.
  * Each output may be NULL.  veto_threshold >= 0 (0 never vetoes).  S = 0 is a
  * no-op.  Errors: DVP_ERR_INVALID_ARG (null inputs, negative sizes, negative or
- * NaN threshold).  Offsets are not checked on the device.
+ * NaN threshold, min_cov or mean_cov without log_cov).  Offsets are not checked
+ * on the device.
  */
 typedef struct {
   uint32_t struct_size;
@@ -333,6 +350,9 @@ typedef struct {
   int32_t *n_zero_weight;
   uint8_t *veto;
   void *stream;
+  const float *log_cov;
+  float *min_cov;
+  float *mean_cov;
 } dvp_sequence_args;
 
 int dvp_sequence_aggregate(const dvp_sequence_args *args);
@@ -384,8 +404,10 @@ int dvp_monitor(const dvp_monitor_args *args);
  * `panel_rows` = 0 selects 128 here.  The call itself allocates and frees
  * nothing, on the device or through any library.
  *
- * Limit: the workspace the arguments need (dvp_workspace_bytes with the same
- * panel_rows; roughly (2 H + 6 panel_rows) V + 2 H T bytes) must fit in
+ * Limit: the workspace the arguments need (dvp_workspace_bytes with the
+ * panel_rows this entry uses: pass panel_rows = 128 to that query when you pass 0
+ * here, since 0 means up to 4096 there; roughly (2 H + 6 panel_rows) V + 2 H T
+ * bytes) must fit in
  * DVP_STATIC_WORKSPACE_BYTES, e.g. H = 1024, V = 8192, any T up to a few
  * thousand.  Larger problems return DVP_ERR_WORKSPACE and launch nothing.
  * Other errors are those of dvp_fused_lmhead_forward_backward;
@@ -401,9 +423,21 @@ int dvp_monitor(const dvp_monitor_args *args);
  * instance on different streams) race on it and corrupt each other; issue such
  * calls on one stream, or order them yourself.  After the stream has finished,
  * nothing in the array is needed any more.
+ *
+ * Status: the ordinary entry point reports a tensor-core kernel that gave up
+ * waiting through the first word of the caller's workspace.  Here the caller
+ * never sees the workspace, so that word is read with
+ * dvp_static_workspace_status: it waits for all work on the current device (it
+ * synchronises), then copies the word of the last call on this device to
+ * *status_out (a host pointer): 0 = every kernel finished, non-zero = results of
+ * that call are invalid.  It allocates nothing either.  Errors:
+ * DVP_ERR_INVALID_ARG (NULL), DVP_ERR_CUDA.  Without this call a wait that ran
+ * out would go unnoticed (the entry point itself still returns DVP_OK, as
+ * launches are asynchronous).
  */
 #define DVP_STATIC_WORKSPACE_BYTES (32u * 1024u * 1024u)
 int dvp_fused_lmhead_forward_backward_static(const dvp_fused_args *args);
+int dvp_static_workspace_status(uint32_t *status_out);
 
 /*
  * dvp_gemm_tn -- the tensor-core contraction the fused entry point is built on,

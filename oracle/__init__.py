@@ -106,6 +106,13 @@ def _load():
         lib.dvp_oracle_side_grad.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                              ctypes.c_double, ctypes.c_void_p, ctypes.c_void_p]
         lib.dvp_oracle_side_grad.restype = None
+        lib.dvp_oracle_side_given_set.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                                  ctypes.c_void_p, ctypes.c_void_p]
+        lib.dvp_oracle_side_given_set.restype = None
+        lib.dvp_oracle_side_grad_given_set.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                                       ctypes.c_double, ctypes.c_void_p, ctypes.c_void_p,
+                                                       ctypes.c_void_p]
+        lib.dvp_oracle_side_grad_given_set.restype = None
         lib.dvp_oracle_log_ratio.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
         lib.dvp_oracle_log_ratio.restype = ctypes.c_double
         lib.dvp_oracle_token_weight.argtypes = [ctypes.c_double, ctypes.c_int, ctypes.c_double, ctypes.c_double]
@@ -248,10 +255,17 @@ class FusedResult:
     d_w: np.ndarray       # [V, H] float64
 
 
+def fused_logits(hidden_bf16: np.ndarray, w_bf16: np.ndarray) -> np.ndarray:
+    """z = h W^T in float64 from bfloat16 bit patterns: the training logits of the LM-head
+    composition, which never round."""
+    return _bf16_bits_to_f64(hidden_bf16) @ _bf16_bits_to_f64(w_bf16).T
+
+
 def dvp_fused_lmhead(hidden_bf16: np.ndarray, w_bf16: np.ndarray, infer_bf16: np.ndarray,
                      ids: np.ndarray, rho: float, upstream: np.ndarray, threads: int = 1,
                      weight_kind: int = WEIGHT_NONE, weight_lo: float = 0.0,
-                     weight_hi: float = float("inf")) -> FusedResult:
+                     weight_hi: float = float("inf"), logits: np.ndarray | None = None,
+                     train_set: np.ndarray | None = None) -> FusedResult:
     """LM-head composition: z = h W^T, then the row computation on z, then the
     chain rule of Prop. 5.6 part 2 through the linear head:
     dH = G W and dW = G^T h with G = dL/dz.
@@ -259,12 +273,19 @@ def dvp_fused_lmhead(hidden_bf16: np.ndarray, w_bf16: np.ndarray, infer_bf16: np
     hidden [T, H], w [V, H] and infer logits [T, V] are bfloat16 bit patterns
     (uint16).  Train logits are taken in float64, so they never round.  With a
     ``weight_kind`` each token's upstream gradient is multiplied by its importance
-    weight (``dvp_oracle_token_weight``), held constant.
+    weight (``dvp_oracle_token_weight``), held constant.  ``logits`` hands in a
+    ``fused_logits`` result computed before.  ``train_set`` ([T, V] bytes) supplies
+    the training safe set instead of deriving it (``dvp_oracle_side_given_set``):
+    the set of Def. 5.1 is fixed only up to tokens within rounding distance of the
+    threshold when the logits themselves come out of rounded arithmetic.
     """
     h = _bf16_bits_to_f64(hidden_bf16)
     w = _bf16_bits_to_f64(w_bf16)
-    z = h @ w.T
+    z = h @ w.T if logits is None else logits
     zi = _bf16_bits_to_f64(infer_bf16)
+    if train_set is not None:
+        train_set = np.ascontiguousarray(train_set, dtype=np.uint8)
+        assert train_set.shape == z.shape
     T, V = z.shape
     # The C rows read float32 or 16-bit storage; float64 logits go through the
     # same per-row functions one row at a time.
@@ -283,7 +304,10 @@ def dvp_fused_lmhead(hidden_bf16: np.ndarray, w_bf16: np.ndarray, infer_bf16: np
         zit = np.ascontiguousarray(zi[t])
         pt = side_t.ctypes.data + t * step
         pi = side_i.ctypes.data + t * step
-        lib.dvp_oracle_side(zt.ctypes.data, V, int(ids[t]), log_rho, pt, None)
+        if train_set is None:
+            lib.dvp_oracle_side(zt.ctypes.data, V, int(ids[t]), log_rho, pt, None)
+        else:
+            lib.dvp_oracle_side_given_set(zt.ctypes.data, V, int(ids[t]), train_set[t].ctypes.data, pt)
         lib.dvp_oracle_side(zit.ctypes.data, V, int(ids[t]), log_rho, pi, None)
         log_ratio[t] = lib.dvp_oracle_log_ratio(pt, pi)
         g = float(up[t])
@@ -292,7 +316,11 @@ def dvp_fused_lmhead(hidden_bf16: np.ndarray, w_bf16: np.ndarray, infer_bf16: np
                                                     float(weight_hi))
             if not np.isnan(weight[t]):
                 g *= float(weight[t])
-        lib.dvp_oracle_side_grad(zt.ctypes.data, V, int(ids[t]), g, pt, grad.ctypes.data + t * V * 8)
+        if train_set is None:
+            lib.dvp_oracle_side_grad(zt.ctypes.data, V, int(ids[t]), g, pt, grad.ctypes.data + t * V * 8)
+        else:
+            lib.dvp_oracle_side_grad_given_set(zt.ctypes.data, V, int(ids[t]), g, train_set[t].ctypes.data, pt,
+                                               grad.ctypes.data + t * V * 8)
     rows = Result(train=_side(side_t, None), infer=_side(side_i, None), log_ratio=log_ratio,
                   grad=grad, threads=1, weight=weight if weight_kind != WEIGHT_NONE else None)
     return FusedResult(rows=rows, logits=z, d_hidden=grad @ w, d_w=grad.T @ h)
@@ -373,6 +401,23 @@ def dvp_sequences(log_ratio: np.ndarray, seq_offsets: np.ndarray, veto_threshold
                                  out.n_valid.ctypes.data, out.n_zero_weight.ctypes.data,
                                  out.veto.ctypes.data)
     return out
+
+
+def dvp_coverage(log_cov: np.ndarray, seq_offsets: np.ndarray):
+    """Per sequence: min and mean over its states of the coverage Z = e^{ln Z}
+    (Def. 5.2; the minimum is the Z_min of the bias bound of Prop. 5.5)."""
+    lib = _load()
+    lc = np.ascontiguousarray(log_cov, dtype=np.float64)
+    off = np.ascontiguousarray(seq_offsets, dtype=np.int64)
+    S = len(off) - 1
+    assert S >= 0 and (S == 0 or (off[0] >= 0 and off[-1] <= len(lc) and (np.diff(off) >= 0).all()))
+    lo, mean = np.zeros(S), np.zeros(S)
+    lib.dvp_oracle_coverage.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
+                                        ctypes.c_void_p]
+    lib.dvp_oracle_coverage.restype = None
+    if S > 0:
+        lib.dvp_oracle_coverage(lc.ctypes.data, off.ctypes.data, S, lo.ctypes.data, mean.ctypes.data)
+    return lo, mean
 
 
 _LISTING_DTYPE = np.dtype([("max", "f8"), ("lse_full", "f8"), ("lse_masked", "f8"), ("logp_masked", "f8"),

@@ -173,6 +173,61 @@ void dvp_oracle_side_grad(const double *z, int64_t V, int64_t a, double g,
 }
 
 /*
+ * The same statistics with the safe set supplied instead of derived from a
+ * threshold: Def. 5.2 and Prop. 5.4 take V_S as given (set: V bytes, 1 where k is
+ * in the set).  For logits that exist only up to rounding (the LM-head variant on
+ * tensor cores) the set of Def. 5.1 is fixed only up to tokens whose logit sits
+ * within rounding distance of the threshold; this form states what every other
+ * quantity must be for whichever of those sets was taken.  With the set that
+ * dvp_oracle_side itself derives it returns the same numbers.  tau is NaN.
+ */
+void dvp_oracle_side_given_set(const double *z, int64_t V, int64_t a, const uint8_t *set,
+                               oracle_side *out) {
+  double m = -INFINITY;
+  for (int64_t k = 0; k < V; ++k)
+    if (z[k] > m) m = z[k];
+  nsum all = {0, 0}, safe = {0, 0}, safe_x = {0, 0};
+  int64_t n = 0;
+  for (int64_t k = 0; k < V; ++k) {
+    const double e = exp(z[k] - m);
+    nsum_add(&all, e);
+    if (set[k]) {
+      nsum_add(&safe, e);
+      if (k != a) nsum_add(&safe_x, e);
+      ++n;
+    }
+  }
+  const double s = nsum_value(&all), s_safe = nsum_value(&safe);
+  out->max = m;
+  out->tau = NAN;
+  out->lse = m + log(s);
+  out->lse_safe = m + log(s_safe);
+  out->log_cov = log(s_safe) - log(s);
+  out->sum_safe = s_safe;
+  out->sum_safe_x = nsum_value(&safe_x);
+  out->count = n;
+  if (a >= 0 && a < V) {
+    out->member = set[a] != 0;
+    out->logp = (z[a] - m) - log(s);
+    out->logp_mp = out->member ? (z[a] - m) - log(s_safe) : -INFINITY;
+  } else {
+    out->member = 0;
+    out->logp = NAN;
+    out->logp_mp = NAN;
+  }
+}
+
+void dvp_oracle_side_grad_given_set(const double *z, int64_t V, int64_t a, double g,
+                                    const uint8_t *set, const oracle_side *st, double *grad) {
+  if (a < 0 || a >= V || !st->member) {
+    for (int64_t k = 0; k < V; ++k) grad[k] = 0.0;
+    return;
+  }
+  for (int64_t k = 0; k < V; ++k) grad[k] = set[k] ? -g * exp(z[k] - st->lse_safe) : 0.0;
+  grad[a] = g * (st->sum_safe_x / st->sum_safe);
+}
+
+/*
  * Per-token log-ratio r = ln pi^mp_train(a) - ln pi^mp_infer(a).
  * a outside the training set: the importance ratio is zero (remark after
  * Thm. 5.3), r = -inf whatever the inference side says.  a inside the
@@ -423,6 +478,27 @@ void dvp_oracle_sequences(const double *log_ratio, const int64_t *off, int64_t S
     n_valid[s] = valid;
     n_zero_weight[s] = zero;
     veto[s] = (uint8_t)vetoed;
+  }
+}
+
+/*
+ * Coverage statistics of a sequence of states: Z_t = e^{ln Z_t} (Def. 5.2), its
+ * minimum over the sequence (the Z_min of Prop. 5.5's bound
+ * |J_mp - J| <= R_max T (1 - Z_min)) and its mean.  Empty sequence: +inf and NaN.
+ */
+void dvp_oracle_coverage(const double *log_cov, const int64_t *off, int64_t S, double *min_cov,
+                         double *mean_cov) {
+  for (int64_t s = 0; s < S; ++s) {
+    nsum acc = {0, 0};
+    double lo = INFINITY;
+    for (int64_t t = off[s]; t < off[s + 1]; ++t) {
+      const double z = exp(log_cov[t]);
+      if (z < lo) lo = z;
+      nsum_add(&acc, z);
+    }
+    const int64_t n = off[s + 1] - off[s];
+    min_cov[s] = lo;
+    mean_cov[s] = n > 0 ? nsum_value(&acc) / (double)n : NAN;
   }
 }
 

@@ -27,10 +27,11 @@ DVP_WEIGHT_NONE, DVP_WEIGHT_RATIO, DVP_WEIGHT_TRUNCATE, DVP_WEIGHT_MASK = 0, 1, 
 
 EXPORTS = ("dvp_forward", "dvp_backward", "dvp_fused_lmhead_forward_backward",
            "dvp_fused_lmhead_forward_backward_static", "dvp_sequence_aggregate", "dvp_monitor", "dvp_gemm_tn",
-           "dvp_workspace_bytes", "dvp_status_string", "dvp_version", "dvp_row_wait_status")
+           "dvp_workspace_bytes", "dvp_status_string", "dvp_version", "dvp_row_wait_status",
+           "dvp_static_workspace_status")
 
 _DTYPES = {torch.float32: DVP_F32, torch.bfloat16: DVP_BF16, torch.float16: DVP_F16}
-_SIDE_FIELDS = ("max", "lse", "lse_safe", "logp", "logp_mp", "comp_mp", "count", "mask")
+_SIDE_FIELDS = ("max", "lse", "lse_safe", "logp", "logp_mp", "comp_mp", "count", "mask", "log_cov")
 
 
 class DvpError(RuntimeError):
@@ -153,6 +154,9 @@ class SequenceArgs(ctypes.Structure):
         ("n_zero_weight", ctypes.c_void_p),
         ("veto", ctypes.c_void_p),
         ("stream", ctypes.c_void_p),
+        ("log_cov", ctypes.c_void_p),
+        ("min_cov", ctypes.c_void_p),
+        ("mean_cov", ctypes.c_void_p),
     ]
 
 
@@ -210,6 +214,8 @@ def load_library() -> ctypes.CDLL:
         lib.dvp_version.restype = ctypes.c_int
         lib.dvp_row_wait_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
         lib.dvp_row_wait_status.restype = ctypes.c_int
+        lib.dvp_static_workspace_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
+        lib.dvp_static_workspace_status.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -237,7 +243,7 @@ def _check_matrix(name: str, x: torch.Tensor):
 
 def _side(device, T: int, V: int, want_mask: bool):
     o = SimpleNamespace()
-    for n in ("max", "lse", "lse_safe", "logp", "logp_mp", "comp_mp"):
+    for n in ("max", "lse", "lse_safe", "logp", "logp_mp", "comp_mp", "log_cov"):
         setattr(o, n, torch.empty(T, dtype=torch.float32, device=device))
     o.count = torch.empty(T, dtype=torch.int32, device=device)
     o.mask = torch.empty(T, (V + 31) // 32, dtype=torch.int32, device=device) if want_mask else None
@@ -413,20 +419,9 @@ def dvp_workspace_bytes(entry_point: int, args: ctypes.Structure) -> int:
     return int(load_library().dvp_workspace_bytes(int(entry_point), ctypes.byref(args)))
 
 
-def dvp_fused_lmhead_forward_backward(hidden: torch.Tensor, w_vocab: torch.Tensor, ids: torch.Tensor,
-                                      rho: float, upstream: torch.Tensor, *,
-                                      infer_logits: torch.Tensor | None = None,
-                                      d_w: torch.Tensor | None = None, accumulate_dw: bool = False,
-                                      panel_rows: int = 0, workspace: torch.Tensor | None = None,
-                                      stream=None, weight_kind: int = DVP_WEIGHT_NONE,
-                                      weight_lo: float = 0.0, weight_hi: float = 1.0):
-    """Pruned log-probabilities and gradients with respect to ``hidden`` and
-    ``w_vocab`` with the training logits hidden x w_vocab^T produced panel by
-    panel inside the library and never stored as a [T, V] matrix.  With
-    ``weight_kind`` (truncate or mask, finite ``weight_hi``) each token's upstream
-    gradient is multiplied by its importance weight; the weights come back as
-    ``weight``."""
-    lib = load_library()
+def _fused_args(hidden, w_vocab, ids, rho, upstream, infer_logits, d_w, accumulate_dw, panel_rows, stream,
+                want_mask=False):
+    """Marshals the arguments both fused entry points share; creates the output tensors."""
     _check_matrix("hidden", hidden)
     _check_matrix("w_vocab", w_vocab)
     T, H = hidden.shape
@@ -441,7 +436,7 @@ def dvp_fused_lmhead_forward_backward(hidden: torch.Tensor, w_vocab: torch.Tenso
     a.ld_hidden, a.ld_w = hidden.stride(0), w_vocab.stride(0)
     a.hidden, a.w_vocab, a.ids, a.upstream = _ptr(hidden), _ptr(w_vocab), _ptr(ids), _ptr(upstream)
     res = SimpleNamespace(infer=None, log_ratio=None)
-    res.train, a.train = _side(dev, T, V, False)
+    res.train, a.train = _side(dev, T, V, want_mask)
     res.flags = torch.empty(T, dtype=torch.uint8, device=dev)
     a.flags = _ptr(res.flags)
     if infer_logits is not None:
@@ -458,16 +453,35 @@ def dvp_fused_lmhead_forward_backward(hidden: torch.Tensor, w_vocab: torch.Tenso
     a.d_w, a.ld_dw = _ptr(res.d_w), res.d_w.stride(0)
     a.accumulate_dw = int(accumulate_dw)
     a.panel_rows = int(panel_rows)
+    a.stream = _stream(stream)
+    return a, res
+
+
+def dvp_fused_lmhead_forward_backward(hidden: torch.Tensor, w_vocab: torch.Tensor, ids: torch.Tensor,
+                                      rho: float, upstream: torch.Tensor, *,
+                                      infer_logits: torch.Tensor | None = None,
+                                      d_w: torch.Tensor | None = None, accumulate_dw: bool = False,
+                                      panel_rows: int = 0, workspace: torch.Tensor | None = None,
+                                      stream=None, weight_kind: int = DVP_WEIGHT_NONE,
+                                      weight_lo: float = 0.0, weight_hi: float = 1.0, want_mask: bool = False):
+    """Pruned log-probabilities and gradients with respect to ``hidden`` and
+    ``w_vocab`` with the training logits hidden x w_vocab^T produced panel by
+    panel inside the library and never stored as a [T, V] matrix.  With
+    ``weight_kind`` (truncate or mask, finite ``weight_hi``) each token's upstream
+    gradient is multiplied by its importance weight; the weights come back as
+    ``weight``.  ``want_mask`` asks for the packed training safe set."""
+    lib = load_library()
+    a, res = _fused_args(hidden, w_vocab, ids, rho, upstream, infer_logits, d_w, accumulate_dw, panel_rows,
+                         stream, want_mask)
     need = dvp_workspace_bytes(DVP_ENTRY_FUSED_LMHEAD, a)
     if workspace is None:
-        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=hidden.device)
     res.workspace = workspace
     a.workspace, a.workspace_bytes = _ptr(workspace), workspace.numel() * workspace.element_size()
-    a.stream = _stream(stream)
     a.weight_kind = int(weight_kind)
     if weight_kind != DVP_WEIGHT_NONE:
         a.weight_lo, a.weight_hi = float(weight_lo), float(weight_hi)
-        res.weight = torch.empty(T, dtype=torch.float32, device=dev)
+        res.weight = torch.empty(hidden.shape[0], dtype=torch.float32, device=hidden.device)
         a.weight_out = _ptr(res.weight)
     st = lib.dvp_fused_lmhead_forward_backward(ctypes.byref(a))
     if st != DVP_OK:
@@ -489,51 +503,35 @@ def dvp_fused_lmhead_forward_backward_static(hidden: torch.Tensor, w_vocab: torc
     Problems whose workspace would not fit raise ``DvpError`` with
     ``DVP_ERR_WORKSPACE``.  All calls on a GPU share that one array, so calls
     that could overlap on the GPU (different streams) must be ordered by the
-    caller.  Make the first call on each device outside any stream capture."""
+    caller.  Make the first call on each device outside any stream capture.
+    ``dvp_static_workspace_status`` reads the status word of the last call."""
     lib = load_library()
-    _check_matrix("hidden", hidden)
-    _check_matrix("w_vocab", w_vocab)
-    T, H = hidden.shape
-    V = w_vocab.shape[0]
-    dev = hidden.device
-    if hidden.dtype != torch.bfloat16 or w_vocab.dtype != torch.bfloat16:
-        raise TypeError("hidden and w_vocab must be bfloat16")
-    a = FusedArgs()
-    a.struct_size = ctypes.sizeof(FusedArgs)
-    a.id_dtype = _id_dtype(ids)
-    a.T, a.H, a.V, a.rho = T, H, V, float(rho)
-    a.ld_hidden, a.ld_w = hidden.stride(0), w_vocab.stride(0)
-    a.hidden, a.w_vocab, a.ids, a.upstream = _ptr(hidden), _ptr(w_vocab), _ptr(ids), _ptr(upstream)
-    res = SimpleNamespace(infer=None, log_ratio=None)
-    res.train, a.train = _side(dev, T, V, False)
-    res.flags = torch.empty(T, dtype=torch.uint8, device=dev)
-    a.flags = _ptr(res.flags)
-    if infer_logits is not None:
-        _check_matrix("infer_logits", infer_logits)
-        if infer_logits.dtype != torch.bfloat16:
-            raise TypeError("infer_logits must be bfloat16")
-        a.infer_logits, a.ld_infer = _ptr(infer_logits), infer_logits.stride(0)
-        res.infer, a.infer = _side(dev, T, V, False)
-        res.log_ratio = torch.empty(T, dtype=torch.float32, device=dev)
-        a.log_ratio = _ptr(res.log_ratio)
-    res.d_hidden = torch.empty(T, H, dtype=torch.float32, device=dev)
-    res.d_w = d_w if d_w is not None else torch.empty(V, H, dtype=torch.float32, device=dev)
-    a.d_hidden, a.ld_dh = _ptr(res.d_hidden), res.d_hidden.stride(0)
-    a.d_w, a.ld_dw = _ptr(res.d_w), res.d_w.stride(0)
-    a.accumulate_dw = int(accumulate_dw)
-    a.panel_rows = int(panel_rows)
-    a.stream = _stream(stream)
+    a, res = _fused_args(hidden, w_vocab, ids, rho, upstream, infer_logits, d_w, accumulate_dw, panel_rows,
+                         stream)
     st = lib.dvp_fused_lmhead_forward_backward_static(ctypes.byref(a))
     if st != DVP_OK:
         raise DvpError(st, "dvp_fused_lmhead_forward_backward_static")
     return res
 
 
+def dvp_static_workspace_status() -> int:
+    """Waits for the current device and returns the status word that the tensor-core kernels of
+    the last ``dvp_fused_lmhead_forward_backward_static`` call left in the built-in workspace:
+    0 when every kernel finished, non-zero when one gave up waiting (results invalid)."""
+    out = ctypes.c_uint32(0)
+    st = load_library().dvp_static_workspace_status(ctypes.byref(out))
+    if st != DVP_OK:
+        raise DvpError(st, "dvp_static_workspace_status")
+    return int(out.value)
+
+
 def dvp_sequence_aggregate(log_ratio: torch.Tensor, seq_offsets: torch.Tensor,
-                           veto_threshold: float = 1e-4, stream=None):
+                           veto_threshold: float = 1e-4, stream=None, log_cov: torch.Tensor | None = None):
     """Per-sequence sum and minimum of the token log-ratios, token counts and the
     veto flag (Sec. 4.4, Thm. 5.3, App. A protocol 5).  ``seq_offsets`` is an
-    int64 device tensor of S + 1 non-decreasing token offsets."""
+    int64 device tensor of S + 1 non-decreasing token offsets.  With ``log_cov``
+    (ln Z per token from ``dvp_forward``) also the minimum and the mean of the
+    coverage Z over each sequence (Def. 5.2; the Z_min of Prop. 5.5)."""
     lib = load_library()
     if log_ratio.dtype != torch.float32 or seq_offsets.dtype != torch.int64:
         raise TypeError("log_ratio must be float32 and seq_offsets int64")
@@ -553,6 +551,12 @@ def dvp_sequence_aggregate(log_ratio: torch.Tensor, seq_offsets: torch.Tensor,
     a.seq_log_ratio, a.min_log_ratio = _ptr(res.seq_log_ratio), _ptr(res.min_log_ratio)
     a.n_valid, a.n_zero_weight, a.veto = _ptr(res.n_valid), _ptr(res.n_zero_weight), _ptr(res.veto)
     a.stream = _stream(stream)
+    if log_cov is not None:
+        if log_cov.dtype != torch.float32 or log_cov.numel() != log_ratio.numel():
+            raise TypeError("log_cov must be float32 with one entry per token")
+        res.min_cov = torch.empty(S, dtype=torch.float32, device=dev)
+        res.mean_cov = torch.empty(S, dtype=torch.float32, device=dev)
+        a.log_cov, a.min_cov, a.mean_cov = _ptr(log_cov), _ptr(res.min_cov), _ptr(res.mean_cov)
     st = lib.dvp_sequence_aggregate(ctypes.byref(a))
     if st != DVP_OK:
         raise DvpError(st, "dvp_sequence_aggregate")

@@ -22,7 +22,7 @@ bool mode_ok(uint32_t mode, float mask_value) {
 
 bool side_empty(const dvp_side_out &o) {
   return !o.max && !o.lse && !o.lse_safe && !o.logp && !o.logp_mp && !o.comp_mp && !o.count &&
-         !o.mask;
+         !o.mask && !o.log_cov;
 }
 
 double log_of_rho(double rho) { return rho > 0.0 ? std::log(rho) : -HUGE_VAL; }
@@ -135,6 +135,6 @@ const char *dvp_status_string(int status) {
   }
 }
 
-int dvp_version(void) { return 100; }
+int dvp_version(void) { return 200; }
 
 }  // extern "C"

@@ -334,6 +334,8 @@ __device__ __forceinline__ float threshold_of(float m, double log_rho, int mode)
 struct SideStats {
   float m;       // row max
   double lse;    // ln sum_k e^{z_k}
+  double sum_c;  // the full sum as 2^sum_c * sum_s (base 2, exponents scaled by kLog2e as the safe sum is)
+  float sum_s;
   float s_x;     // sum over the safe set of e^{z_k - m}, without the sampled token
   float e_a;     // e^{z_a - m} when a is in the safe set, else 0
   float s_mask;  // mass of the masked tokens, (V - n) e^{mask_value - m}; 0 without a finite mask
@@ -389,6 +391,12 @@ __device__ __forceinline__ float finish_side(const dvp_side_out &o, long long t,
   if (o.logp_mp) o.logp_mp[t] = logp_mp;
   if (o.comp_mp) o.comp_mp[t] = comp;
   if (o.count) o.count[t] = st.n;
+  if (o.log_cov) {
+    // ln Z = ln(safe sum / full sum), both sums of 2^{z l}; one thread, so double logarithms cost nothing
+    const double safe2 = (double)st.m * (double)kLog2e + log2((double)st.s_x + (double)st.e_a);
+    const double full2 = st.sum_c + log2((double)st.sum_s);
+    o.log_cov[t] = (float)fmin(0.0, 0.6931471805599453094 * (safe2 - full2));
+  }
   return logp_mp;
 }
 

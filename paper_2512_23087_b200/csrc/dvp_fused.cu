@@ -172,6 +172,7 @@ dvp_side_out offset_side(const dvp_side_out &o, long long r0, long long words) {
   if (r.logp_mp) r.logp_mp += r0;
   if (r.comp_mp) r.comp_mp += r0;
   if (r.count) r.count += r0;
+  if (r.log_cov) r.log_cov += r0;
   if (r.mask) r.mask += r0 * words;
   return r;
 }
@@ -382,6 +383,14 @@ int dvp_fused_lmhead_forward_backward_static(const dvp_fused_args *a) {
   b.workspace = ptr;
   b.workspace_bytes = kStaticWorkspaceBytes;
   return dvp_fused_lmhead_forward_backward(&b);
+}
+
+int dvp_static_workspace_status(uint32_t *status_out) {
+  if (!status_out) return DVP_ERR_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return DVP_ERR_CUDA;
+  // the status is the first word of the workspace, here of the built-in array
+  return cudaMemcpyFromSymbol(status_out, g_static_workspace, sizeof(uint32_t)) == cudaSuccess ? DVP_OK
+                                                                                              : DVP_ERR_CUDA;
 }
 
 }  // extern "C"

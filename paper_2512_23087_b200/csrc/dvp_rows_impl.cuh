@@ -436,6 +436,8 @@ __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int off, i
   SideStats st;
   st.m = all.m;
   st.lse = lse_from_logsum(all);
+  st.sum_c = (double)all.c;
+  st.sum_s = all.s;
   st.tau = threshold_of<TIn>(all.m, log_rho, mode);
   const bool has_a = a >= 0 && a < V;
   st.z_a = has_a ? Storage<TIn>::widen(row[a]) : 0.f;
@@ -629,6 +631,8 @@ __device__ __forceinline__ SideStats row_stats_scalar(const TIn *row, long long 
   SideStats st;
   st.m = all.m;
   st.lse = (double)all.m + (double)logf(all.s);
+  st.sum_c = (double)all.m * (double)kLog2e;
+  st.sum_s = all.s;
   st.tau = threshold_of<TIn>(all.m, log_rho, mode);
   const bool has_a = a >= 0 && a < V;
   st.z_a = has_a ? Storage<TIn>::widen(row[a]) : 0.f;

@@ -473,6 +473,8 @@ __device__ __forceinline__ SideStats consume_side(const TIn *row, TGrad *grow, f
   SideStats st;
   st.m = all.m;
   st.lse = lse_from_logsum(all);
+  st.sum_c = (double)all.c;
+  st.sum_s = all.s;
   st.tau = threshold_of<TIn>(all.m, p.log_rho, p.mode);
   st.z_a = z_a;
   st.member = has_a && z_a >= st.tau;

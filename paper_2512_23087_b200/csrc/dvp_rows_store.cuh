@@ -391,6 +391,8 @@ __device__ __forceinline__ SideStats side_stats_cs(const TIn *row, const TIn *ne
   SideStats st;
   st.m = all.m;
   st.lse = lse_from_logsum(all);
+  st.sum_c = (double)all.c;
+  st.sum_s = all.s;
   st.tau = threshold_of<TIn>(all.m, p.log_rho, p.mode);
   st.z_a = z_a;
   st.member = has_a && z_a >= st.tau;
@@ -550,6 +552,7 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel_cs(const Row
       o.logp_mp = is_train ? p.out_t.logp_mp : p.out_i.logp_mp;
       o.comp_mp = is_train ? p.out_t.comp_mp : p.out_i.comp_mp;
       o.count = is_train ? p.out_t.count : p.out_i.count;
+      o.log_cov = is_train ? p.out_t.log_cov : p.out_i.log_cov;
       o.mask = nullptr;
       lp = finish_side(o, t, s, has_id, bad_id);
     }

@@ -13,14 +13,18 @@ namespace dvp {
 
 struct SeqPartial {
   double sum;
+  double cov_sum;  // sum of the coverages Z_t = e^{ln Z_t}
   float lo;
+  float cov_lo;
   int valid, zero, pinf, veto;
 };
 
 __device__ __forceinline__ SeqPartial seq_combine(const SeqPartial &a, const SeqPartial &b) {
   SeqPartial r;
   r.sum = a.sum + b.sum;
+  r.cov_sum = a.cov_sum + b.cov_sum;
   r.lo = fminf(a.lo, b.lo);
+  r.cov_lo = fminf(a.cov_lo, b.cov_lo);
   r.valid = a.valid + b.valid;
   r.zero = a.zero + b.zero;
   r.pinf = a.pinf | b.pinf;
@@ -31,7 +35,9 @@ __device__ __forceinline__ SeqPartial seq_combine(const SeqPartial &a, const Seq
 __device__ __forceinline__ SeqPartial seq_shfl(const SeqPartial &v, int o) {
   SeqPartial r;
   r.sum = __shfl_xor_sync(0xffffffffu, v.sum, o);
+  r.cov_sum = __shfl_xor_sync(0xffffffffu, v.cov_sum, o);
   r.lo = __shfl_xor_sync(0xffffffffu, v.lo, o);
+  r.cov_lo = __shfl_xor_sync(0xffffffffu, v.cov_lo, o);
   r.valid = __shfl_xor_sync(0xffffffffu, v.valid, o);
   r.zero = __shfl_xor_sync(0xffffffffu, v.zero, o);
   r.pinf = __shfl_xor_sync(0xffffffffu, v.pinf, o);
@@ -44,11 +50,16 @@ __global__ void __launch_bounds__(256) dvp_sequence_kernel(const dvp_sequence_ar
   __shared__ SeqPartial part[8];
   const long long s = blockIdx.x;
   const long long t0 = a.seq_offsets[s], t1 = a.seq_offsets[s + 1];
-  SeqPartial acc = {0.0, -kNegInf, 0, 0, 0, 0};
+  SeqPartial acc = {0.0, 0.0, -kNegInf, -kNegInf, 0, 0, 0, 0};
   // each thread takes a contiguous slice so that the order of the sum is fixed
   const long long n = t1 - t0, per = (n + blockDim.x - 1) / blockDim.x;
   const long long b = t0 + per * threadIdx.x, e = b + per < t1 ? b + per : t1;
   for (long long t = b; t < e; ++t) {
+    if (a.log_cov) {  // the coverage of a state does not depend on the sampled token
+      const float z = expf(a.log_cov[t]);
+      acc.cov_sum += (double)z;
+      acc.cov_lo = fminf(acc.cov_lo, z);
+    }
     const float r = a.log_ratio[t];
     if (r != r) continue;  // no sampled token
     ++acc.valid;
@@ -79,6 +90,8 @@ __global__ void __launch_bounds__(256) dvp_sequence_kernel(const dvp_sequence_ar
     if (a.n_valid) a.n_valid[s] = r.valid;
     if (a.n_zero_weight) a.n_zero_weight[s] = r.zero;
     if (a.veto) a.veto[s] = (uint8_t)r.veto;
+    if (a.min_cov) a.min_cov[s] = r.cov_lo;
+    if (a.mean_cov) a.mean_cov[s] = n > 0 ? (float)(r.cov_sum / (double)n) : __int_as_float(0x7fc00000);
   }
 }
 
@@ -90,6 +103,7 @@ extern "C" int dvp_sequence_aggregate(const dvp_sequence_args *a) {
   if (!(a->veto_threshold >= 0.0)) return DVP_ERR_INVALID_ARG;
   if (a->S == 0) return DVP_OK;
   if (!a->seq_offsets || !a->log_ratio) return DVP_ERR_INVALID_ARG;
+  if ((a->min_cov || a->mean_cov) && !a->log_cov) return DVP_ERR_INVALID_ARG;
   // e^r < threshold  <=>  r < ln(threshold).  With ln(threshold) rounded up to the next
   // float, "r < log_veto" decides every float r as the real-number comparison does.
   const int positive = a->veto_threshold > 0.0;

@@ -4,13 +4,19 @@ with the fp64 oracle, through the C ABI.
 Membership in the fused variant is decided on bf16 x bf16 products accumulated
 in fp32 by the tensor cores (H/16 accumulation steps, each good to one unit in
 the last place of the running sum), so it cannot be bit-exact against fp64
-logits: rows that hold a logit within (H/16 + 2) 2^-24 max|z| + 1e-6 of the
-threshold are counted and compared on log-probabilities only (their safe-set
-size may differ by at most the number of such logits); every other row is
-compared exactly like the row kernels.
+logits: a logit within (H/16 + 2) 2^-24 max|z| + 1e-6 of the threshold (the
+rounding band) may fall on either side.  The device's packed safe set is
+therefore read back: outside the band it must equal the set of Def. 5.1 on the
+float64 logits bit for bit; inside the band either decision is accepted, and the
+oracle then states what every other quantity must be for the set the device took
+(dvp_oracle_side_given_set).  Against that, every token is compared exactly
+like the row kernels: counts, flags and infinities exact, log-probabilities
+within 1e-4.  How many logits sat in the band, and how many of them the device
+decided the other way, is reported.
 Gradients: per token row of d_hidden and per vocabulary row of d_w,
 ||X - X_oracle||_2 <= 1e-3 ||X_oracle||_2 + 1e-6 * (largest row norm), the second
 term covering rows that are zero up to the float16 grid of the gradient panel.
+d_w is compared on every vocabulary row in every test.
 """
 import numpy as np
 import pytest
@@ -116,72 +122,93 @@ def test_gemm_tn_padded_strides_and_argument_errors():
     assert e.value.status == binding.DVP_ERR_UNSUPPORTED
 
 
-def _check_fused(batch, rho, res, want, V, weight=None):
-    """weight: (kind, lo, hi) of an importance-weighted call; rows whose ratio sits within 5e-4
-    relative of a masking bound (where the weight jumps) are left out of the gradient rows."""
-    rep = {}
-    z = want.logits
-    H = batch.hidden.shape[1]
-    for label, got, side, logits in (("train", res.train, want.rows.train, z),
-                                     ("infer", res.infer, want.rows.infer, None)):
+def _oracle_with_the_devices_set(batch, rho, res, weight=None, rep=None):
+    """The oracle's result for the safe set the device took.  The set of Def. 5.1 is computed
+    on the float64 logits; logits within the rounding band of the threshold may fall on either
+    side on the device, every other logit must agree exactly.  The oracle then states what all
+    other quantities must be for the device's set (dvp_oracle_side_given_set)."""
+    rep = {} if rep is None else rep
+    H, V = batch.hidden.shape[1], batch.w_vocab.shape[0]
+    z = oracle.fused_logits(_bits(batch.hidden), _bits(batch.w_vocab))
+    ids = batch.ids.cpu().numpy()
+    own = oracle.dvp_rows_f64(z, np.where((ids >= 0) & (ids < V), ids, -1), rho, want_mask=True).train
+    width = (H / 16 + 2) * 2.0 ** -24 * np.abs(z).max(axis=1, keepdims=True) + 1e-6
+    band = np.abs(z - own.tau[:, None]) <= width
+    dev_set = parity.unpack_mask(res.train.mask, V)
+    assert np.array_equal(dev_set[~band], own.mask[~band]), "membership differs outside the rounding band"
+    rep["band_tokens"] = rep.get("band_tokens", 0) + int(band.sum())
+    rep["band_rows"] = rep.get("band_rows", 0) + int(band.any(axis=1).sum())
+    rep["band_tokens_decided_otherwise"] = rep.get("band_tokens_decided_otherwise", 0) + \
+        int((dev_set[band] != own.mask[band]).sum())
+    wkw = {} if weight is None else dict(weight_kind=weight[0], weight_lo=weight[1], weight_hi=weight[2])
+    want = oracle.dvp_fused_lmhead(_bits(batch.hidden), _bits(batch.w_vocab), _bits(batch.infer), ids, rho,
+                                   batch.upstream.cpu().numpy().astype(np.float64), logits=z,
+                                   train_set=np.where(band, dev_set, own.mask).astype(np.uint8), **wkw)
+    return want, rep
+
+
+def _rows_close(got, ref, name, rep, rows=None):
+    got = got.cpu().double().numpy() if isinstance(got, torch.Tensor) else got
+    if rows is not None:
+        got, ref = got[rows], ref[rows]
+    num = np.sqrt(((got - ref) ** 2).sum(axis=1))
+    den = np.sqrt((ref ** 2).sum(axis=1))
+    bound = 1e-3 * den + 1e-6 * den.max()
+    assert (num <= bound).all(), f"{name}: worst {np.max(num / np.maximum(den, 1e-300)):.3e}"
+    rep[name] = float(np.max(num / np.maximum(den, 1e-6 * den.max())))
+
+
+def _check_fused(batch, rho, res, want, V, weight=None, rerun=None, d_w_extra=0.0, check_dw=True, rep=None):
+    """Every token against the oracle's result for the device's safe set: counts, flags and
+    infinities exact, log-probabilities within 1e-4, gradient rows within 1e-3 relative L2.
+    weight: (kind, lo, hi) of an importance-weighted call; tokens whose ratio sits within 5e-4
+    relative of a masking bound (where the weight jumps) are left out of the gradient rows, and
+    d_w is then compared on a second call (rerun(upstream)) with their upstream gradient zeroed.
+    d_w_extra is what d_w held before an accumulating call."""
+    rep = {} if rep is None else rep
+    T = len(want.rows.train.count)
+    for label, got, side in (("train", res.train, want.rows.train), ("infer", res.infer, want.rows.infer)):
         if got is None:
             continue
-        if logits is None:
-            logits = batch.infer.detach().cpu().double().numpy()
-        tau = side.tau[:, None]
-        width = (H / 16 + 2) * 2.0 ** -24 * np.abs(logits).max(axis=1, keepdims=True) + 1e-6
-        band = np.abs(logits - tau) <= width
-        band_rows = band.any(axis=1) if label == "train" else np.zeros(len(tau), dtype=bool)
-        ok = ~band_rows
-        rep[f"{label}_band_rows"] = int(band_rows.sum())
-        cnt = got.count.cpu().numpy().astype(np.int64)
-        assert np.array_equal(cnt[ok], side.count[ok]), f"{label}.count"
-        assert (np.abs(cnt - side.count) <= band.sum(axis=1))[band_rows].all()
+        assert np.array_equal(got.count.cpu().numpy().astype(np.int64), side.count), f"{label}.count"
         np.testing.assert_allclose(got.max.cpu().numpy(), side.max, atol=1e-4, rtol=0)
         np.testing.assert_allclose(got.lse.cpu().numpy(), side.lse, atol=1e-4, rtol=0)
         np.testing.assert_allclose(got.lse_safe.cpu().numpy(), side.lse_safe, atol=1e-4, rtol=0)
-        np.testing.assert_allclose(got.logp.cpu().numpy(), side.logp, atol=1e-4, rtol=0)
-        lp = got.logp_mp.cpu().numpy().astype(np.float64)
-        assert np.array_equal(np.isneginf(lp)[ok], np.isneginf(side.logp_mp)[ok])
-        fin = np.isfinite(side.logp_mp) & np.isfinite(lp)
-        assert np.abs(lp[fin] - side.logp_mp[fin]).max() <= 1e-4
-        rep[f"{label}_ok"] = ok
-    ok = rep["train_ok"]
+        np.testing.assert_allclose(got.log_cov.cpu().numpy(), side.log_cov, atol=1e-4, rtol=0)
+        parity._close(got.logp.cpu(), side.logp, 1e-4, f"{label}.logp")
+        parity._close(got.logp_mp.cpu(), side.logp_mp, 1e-4, f"{label}.logp_mp")
     flags = res.flags.cpu().numpy()
-    assert np.array_equal((flags & 1)[ok], want.rows.train.member[ok])
+    assert np.array_equal(flags & 1, want.rows.train.member)
     if res.infer is not None:
         assert np.array_equal((flags >> 1) & 1, want.rows.infer.member)
-        lr = res.log_ratio.cpu().numpy().astype(np.float64)
-        wl = want.rows.log_ratio
-        fin = np.isfinite(wl) & ok
-        assert np.abs(lr[fin] - wl[fin]).max() <= 2e-4
-        assert np.array_equal(np.isinf(lr)[ok], np.isinf(wl)[ok])
-
-    def rows_close(got, ref, name, rows=None):
-        got = got.cpu().double().numpy()
-        if rows is not None:
-            got, ref = got[rows], ref[rows]
-        num = np.sqrt(((got - ref) ** 2).sum(axis=1))
-        den = np.sqrt((ref ** 2).sum(axis=1))
-        bound = 1e-3 * den + 1e-6 * den.max()
-        assert (num <= bound).all(), f"{name}: worst {np.max(num / np.maximum(den, 1e-300)):.3e}"
-        rep[name] = float(np.max(num / np.maximum(den, 1e-6 * den.max())))
-
+        parity._close(res.log_ratio.cpu(), want.rows.log_ratio, 2e-4, "log_ratio")
+    ok = np.ones(T, dtype=bool)
     if weight is not None:
         ratio = np.exp(want.rows.log_ratio)
-        near = np.zeros(len(ratio), dtype=bool)
+        near = np.zeros(T, dtype=bool)
         if weight[0] == oracle.WEIGHT_MASK:
             with np.errstate(invalid="ignore"):
                 near = (np.abs(ratio - weight[1]) <= 5e-4 * weight[1]) | (np.abs(ratio - weight[2]) <= 5e-4 * weight[2])
         rep["near_weight_bound_rows"] = int(near.sum())
-        ok = ok & ~near
+        ok = ~near
         got_w = res.weight.cpu().numpy().astype(np.float64)
         assert np.array_equal(np.isnan(got_w), np.isnan(want.rows.weight))
         assert (np.abs(got_w - want.rows.weight)[ok] <= 2e-4 * np.abs(want.rows.weight[ok]) + 1e-12).all(), "weight"
         rep["zero_weight_rows"] = int((want.rows.weight[ok] == 0).sum())
-    rows_close(res.d_hidden, want.d_hidden, "d_hidden", ok)
+    _rows_close(res.d_hidden, want.d_hidden, "d_hidden", rep, ok)
+    rep["ok_rows"] = ok
+    if not check_dw:
+        return rep
     if ok.all():
-        rows_close(res.d_w, want.d_w, "d_w")
+        _rows_close(res.d_w, want.d_w + d_w_extra, "d_w", rep)
+    else:
+        # the tokens left out contribute G_t^T h_t each: zero their upstream on the device,
+        # take their terms out of the oracle's sum
+        up = batch.upstream.clone()
+        up[torch.from_numpy(~ok).to(up.device)] = 0.0
+        again = rerun(up)
+        h = batch.hidden.detach().cpu().double().numpy()
+        _rows_close(again.d_w, want.d_w - want.rows.grad[~ok].T @ h[~ok] + d_w_extra, "d_w", rep)
     return rep
 
 
@@ -189,21 +216,23 @@ def _run_fused(T, H, V, rho, seed, weight=None, **kw):
     w = inputs.WORKLOADS["c4_fused_lmhead"]
     batch = inputs.make_fused(w, seed=seed, device=DEV, T=T, H=H, V=V)
     wkw = {} if weight is None else dict(weight_kind=weight[0], weight_lo=weight[1], weight_hi=weight[2])
-    res = binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, rho,
-                                                    batch.upstream, infer_logits=batch.infer, **wkw, **kw)
-    torch.cuda.synchronize()
-    assert res.workspace[:4].view(torch.int32).item() == 0, "a tensor-core kernel gave up waiting"
-    want = oracle.dvp_fused_lmhead(_bits(batch.hidden), _bits(batch.w_vocab), _bits(batch.infer),
-                                   batch.ids.cpu().numpy(), rho, batch.upstream.cpu().numpy().astype(np.float64),
-                                   **wkw)
-    return batch, res, want
+
+    def rerun(upstream):
+        r = binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, rho, upstream,
+                                                      infer_logits=batch.infer, want_mask=True, **wkw, **kw)
+        torch.cuda.synchronize()
+        assert r.workspace[:4].view(torch.int32).item() == 0, "a tensor-core kernel gave up waiting"
+        return r
+    res = rerun(batch.upstream)
+    want, rep = _oracle_with_the_devices_set(batch, rho, res, weight)
+    return batch, res, want, rerun
 
 
 @pytest.mark.parametrize("T,H,V,rho", [(200, 256, 3000, 1e-3), (64, 128, 1000, 1e-2), (130, 512, 5008, 1e-4),
                                        (128, 4096, 4096, 1e-3)])
 def test_fused_lmhead_small(T, H, V, rho):
-    batch, res, want = _run_fused(T, H, V, rho, seed=T)
-    _check_fused(batch, rho, res, want, V)
+    batch, res, want, rerun = _run_fused(T, H, V, rho, seed=T)
+    _check_fused(batch, rho, res, want, V, rerun=rerun)
 
 
 @pytest.mark.parametrize("weight", [(oracle.WEIGHT_TRUNCATE, 0.0, 1.004), (oracle.WEIGHT_MASK, 0.985, 1.01)],
@@ -212,8 +241,8 @@ def test_fused_lmhead_small(T, H, V, rho):
 def test_fused_lmhead_importance_weighted(T, H, V, rho, panel, weight):
     """Thm. 5.3 per token through the LM head: the inference rows are swept first, the
     training panels take the weight from them; one panel and several."""
-    batch, res, want = _run_fused(T, H, V, rho, seed=T + 1, weight=weight, panel_rows=panel)
-    rep = _check_fused(batch, rho, res, want, V, weight=weight)
+    batch, res, want, rerun = _run_fused(T, H, V, rho, seed=T + 1, weight=weight, panel_rows=panel)
+    rep = _check_fused(batch, rho, res, want, V, weight=weight, rerun=rerun)
     assert (want.rows.weight != np.exp(want.rows.log_ratio))[np.isfinite(want.rows.log_ratio)].any()   # the bounds do cut
     if weight[0] == oracle.WEIGHT_MASK:
         assert rep["zero_weight_rows"] >= 1
@@ -232,13 +261,11 @@ def test_fused_lmhead_several_panels_and_dw_accumulation():
     d_w = torch.full((V, H), 0.5, device=DEV)
     res = binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, rho,
                                                     batch.upstream, infer_logits=batch.infer,
-                                                    panel_rows=128, d_w=d_w, accumulate_dw=True)
+                                                    panel_rows=128, d_w=d_w, accumulate_dw=True, want_mask=True)
     torch.cuda.synchronize()
     assert res.workspace[:4].view(torch.int32).item() == 0
-    want = oracle.dvp_fused_lmhead(_bits(batch.hidden), _bits(batch.w_vocab), _bits(batch.infer),
-                                   batch.ids.cpu().numpy(), rho, batch.upstream.cpu().numpy().astype(np.float64))
-    want.d_w += 0.5
-    rep = _check_fused(batch, rho, res, want, V)
+    want, rep = _oracle_with_the_devices_set(batch, rho, res)
+    _check_fused(batch, rho, res, want, V, d_w_extra=0.5, rep=rep)
     one = binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, rho,
                                                     batch.upstream, infer_logits=batch.infer)
     torch.cuda.synchronize()
@@ -248,9 +275,76 @@ def test_fused_lmhead_several_panels_and_dw_accumulation():
 
 def test_fused_lmhead_full_vocabulary_rows():
     """V = 151,936 with the LM-head statistics of the benchmark configuration."""
-    batch, res, want = _run_fused(256, 1024, 151936, 1e-3, seed=3)
-    rep = _check_fused(batch, 1e-3, res, want, 151936)
+    batch, res, want, rerun = _run_fused(256, 1024, 151936, 1e-3, seed=3)
+    rep = _check_fused(batch, 1e-3, res, want, 151936, rerun=rerun)
     assert want.rows.train.count.mean() > 1000        # dense safe sets, as in the full configuration
+
+
+def _rows_of(res, sl):
+    """The per-token part of a fused result restricted to the rows `sl`."""
+    from types import SimpleNamespace
+
+    def side(s):
+        if s is None:
+            return None
+        return SimpleNamespace(**{k: (v[sl] if isinstance(v, torch.Tensor) else v) for k, v in vars(s).items()})
+    return SimpleNamespace(train=side(res.train), infer=side(res.infer), log_ratio=res.log_ratio[sl],
+                           flags=res.flags[sl], d_hidden=res.d_hidden[sl], d_w=None,
+                           weight=None if getattr(res, "weight", None) is None else res.weight[sl])
+
+
+@pytest.mark.parametrize("rho", [1e-4, 1e-3])
+def test_fused_lmhead_benchmark_shape_full_panel_and_ragged_panel(rho):
+    """The benchmark configuration's own H = 4096 and V = 151,936 with its default panels: one
+    full panel of 4096 tokens and a ragged one of 128, d_w accumulated across them, K = 4096
+    accumulation steps per logit and K = V in the d_hidden contraction.  The oracle works through
+    the tokens in slabs (float64 logits of a slab are 0.6 GB); per-token outputs and d_hidden are
+    compared on every token, d_w on every vocabulary row, all for the safe sets the device took
+    (which must be the oracle's outside the rounding band; the band's size is printed)."""
+    T, H, V, slab = 4096 + 128, 4096, 151936, 512
+    if _host_memory_available() < 40 << 30:
+        pytest.skip("the float64 oracle of this shape needs about 25 GB of host memory")
+    w = inputs.WORKLOADS["c4_fused_lmhead"]
+    batch = inputs.make_fused(w, seed=11, device=DEV, T=T, H=H, V=V)
+    res = binding.dvp_fused_lmhead_forward_backward(batch.hidden, batch.w_vocab, batch.ids, rho, batch.upstream,
+                                                    infer_logits=batch.infer, want_mask=True)
+    torch.cuda.synchronize()
+    assert res.workspace[:4].view(torch.int32).item() == 0, "a tensor-core kernel gave up waiting"
+    d_w = np.zeros((V, H))
+    rep = {}
+    for r0 in range(0, T, slab):
+        sl = slice(r0, min(T, r0 + slab))
+        sub = inputs.FusedBatch(batch.hidden[sl], batch.w_vocab, batch.infer[sl], batch.ids[sl], batch.upstream[sl])
+        sub_res = _rows_of(res, sl)
+        want, rep = _oracle_with_the_devices_set(sub, rho, sub_res, rep=rep)
+        _check_fused(sub, rho, sub_res, want, V, check_dw=False, rep=rep)
+        d_w += want.d_w
+        del want
+    print(f"rho={rho}: {rep['band_tokens']} logits of {rep['band_rows']} tokens (of {T}) lie within rounding "
+          f"distance of the threshold; the device decided {rep['band_tokens_decided_otherwise']} of them the "
+          f"other way; worst d_hidden row {rep['d_hidden']:.2e}")
+    den = np.sqrt((d_w ** 2).sum(axis=1))
+    num = np.empty(V)
+    for k0 in range(0, V, 16384):                     # vocabulary rows in chunks: no second 5 GB copy
+        ks = slice(k0, min(V, k0 + 16384))
+        num[ks] = np.sqrt(((res.d_w[ks].cpu().double().numpy() - d_w[ks]) ** 2).sum(axis=1))
+    assert (num <= 1e-3 * den + 1e-6 * den.max()).all(), f"d_w: worst {np.max(num / np.maximum(den, 1e-300)):.3e}"
+    assert rep["band_tokens_decided_otherwise"] <= rep["band_tokens"]
+
+
+def _host_memory_available() -> int:
+    """Bytes of host memory this process may still take: the smaller of what the machine has
+    free and what is left under the container's limit."""
+    import psutil
+    avail = psutil.virtual_memory().available
+    try:
+        limit = open("/sys/fs/cgroup/memory.max").read().strip()
+        used = int(open("/sys/fs/cgroup/memory.current").read())
+        if limit != "max":
+            avail = min(avail, int(limit) - used)
+    except OSError:
+        pass
+    return avail
 
 
 def test_fused_argument_errors():

@@ -208,6 +208,37 @@ def test_total_variation_equals_one_minus_coverage():
         assert tv == pytest.approx(1.0 - math.exp(res.train.log_cov[t]), abs=1e-14)
 
 
+def test_coverage_statistics_of_sequences():
+    """dvp_coverage: Z_min and mean Z per sequence.  Pinned through the identity of the proof
+    of Prop. 5.5 (Z = 1 - TV(pi^mp, pi), computed here from the probabilities, not from the
+    oracle's ln Z) and exact summation; empty sequences give +inf and NaN."""
+    rng = np.random.default_rng(31)
+    z = _rows(rng, 37, 11, scale=2.5)
+    res = oracle.dvp_rows_f64(z, np.zeros(37, dtype=np.int64), 0.1, want_mask=True)
+    cov = []
+    for t in range(37):
+        pi = np.exp(z[t] - z[t].max())
+        pi /= pi.sum()
+        safe = res.train.mask[t].astype(bool)
+        pi_mp = np.where(safe, pi / pi[safe].sum(), 0.0)
+        cov.append(1.0 - 0.5 * np.abs(pi_mp - pi).sum())
+    off = np.array([0, 5, 5, 6, 37, 37], dtype=np.int64)
+    lo, mean = oracle.dvp_coverage(res.train.log_cov, off)
+    for s in range(5):
+        seg = cov[off[s]:off[s + 1]]
+        if not seg:
+            assert math.isinf(lo[s]) and lo[s] > 0 and math.isnan(mean[s])
+        else:
+            assert lo[s] == pytest.approx(min(seg), abs=1e-13)
+            assert mean[s] == pytest.approx(math.fsum(seg) / len(seg), abs=1e-13)
+    assert lo[3] < mean[3] < 1.0
+    # the bound of Prop. 5.5 for R_max = 1 is T (1 - Z_min): it grows with the sequence, and a
+    # sequence whose every state keeps the whole vocabulary has bound zero
+    full = oracle.dvp_rows_f64(z, np.zeros(37, dtype=np.int64), 0.0)
+    lo0, mean0 = oracle.dvp_coverage(full.train.log_cov, np.array([0, 37], dtype=np.int64))
+    assert lo0[0] == pytest.approx(1.0, abs=1e-14) and mean0[0] == pytest.approx(1.0, abs=1e-14)
+
+
 @pytest.mark.parametrize("eps_max", [1e-3, 1e-2, 1e-1])
 def test_asymmetric_vulnerability_bound(eps_max):
     """Prop. 4.2.  Its proof bounds |Delta_a| by 2 eps_max (1 - p_a(z_c)) at a
@@ -320,6 +351,53 @@ def test_fused_lmhead_matches_autograd_through_the_head():
     # infer side: an ordinary row pass on the stored bf16 logits
     ref_i = oracle.dvp_rows(bits(zi), ids, rho, dtype=oracle.BF16)
     assert np.array_equal(res.rows.infer.logp_mp, ref_i.train.logp_mp)
+
+
+def test_fused_lmhead_with_a_supplied_safe_set():
+    """dvp_oracle_side_given_set / _grad_given_set through dvp_fused_lmhead(train_set=...):
+    (i) with the set Def. 5.1 derives, the very numbers of the threshold form; (ii) with an
+    arbitrary set (the argmax plus random tokens), pi^mp by explicit renormalisation over that
+    set in probability space (Def. 5.2) and its gradient by autograd through h W^T."""
+    rng = np.random.default_rng(41)
+    T, H, V, rho = 6, 8, 19, 5e-2
+    hb = torch.from_numpy(rng.normal(size=(T, H)).astype(np.float32)).to(torch.bfloat16)
+    wb = torch.from_numpy((rng.normal(size=(V, H)) * 0.5).astype(np.float32)).to(torch.bfloat16)
+    bits = lambda x: x.view(torch.int16).numpy().view(np.uint16)
+    z = oracle.fused_logits(bits(hb), bits(wb))
+    np.testing.assert_allclose(z, hb.double().numpy() @ wb.double().numpy().T, atol=1e-13)
+    zi = torch.from_numpy(z + rng.normal(size=z.shape) * 0.02).to(torch.bfloat16)
+    ids = rng.integers(0, V, size=T)
+    g = rng.normal(size=T)
+    plain = oracle.dvp_fused_lmhead(bits(hb), bits(wb), bits(zi), ids, rho, g)
+    own = (z >= plain.rows.train.tau[:, None]).astype(np.uint8)
+    same = oracle.dvp_fused_lmhead(bits(hb), bits(wb), bits(zi), ids, rho, g, logits=z, train_set=own)
+    for name in ("max", "lse", "lse_safe", "log_cov", "logp", "logp_mp", "sum_safe", "sum_safe_x", "count", "member"):
+        assert np.array_equal(getattr(same.rows.train, name), getattr(plain.rows.train, name), equal_nan=True), name
+    assert np.array_equal(same.d_hidden, plain.d_hidden) and np.array_equal(same.d_w, plain.d_w)
+    assert np.array_equal(same.rows.log_ratio, plain.rows.log_ratio, equal_nan=True)
+    # an arbitrary set
+    chosen = rng.random(size=(T, V)) < 0.4
+    chosen[np.arange(T), z.argmax(1)] = True
+    ids[:4] = [np.flatnonzero(chosen[t])[0] for t in range(4)]     # sampled tokens inside the set
+    ids[4] = np.flatnonzero(~chosen[4])[0]                         # and one outside: zero row
+    res = oracle.dvp_fused_lmhead(bits(hb), bits(wb), bits(zi), ids, rho, g, train_set=chosen.astype(np.uint8))
+    h = hb.to(torch.float64).requires_grad_(True)
+    w = wb.to(torch.float64).requires_grad_(True)
+    pi = torch.softmax(h @ w.t(), dim=-1)
+    sel = torch.from_numpy(chosen)
+    cover = (pi * sel).sum(dim=-1)                                 # Z of Def. 5.2 for the supplied set
+    pi_mp = pi * sel / cover[:, None]
+    picked = pi_mp[torch.arange(T), torch.from_numpy(ids)]
+    inside = picked > 0
+    (torch.log(picked[inside]) * torch.from_numpy(g)[inside]).sum().backward()
+    np.testing.assert_allclose(res.rows.train.logp_mp[inside.numpy()], torch.log(picked[inside]).detach().numpy(),
+                               atol=1e-12)
+    assert np.isneginf(res.rows.train.logp_mp[~inside.numpy()]).all() and not inside[4]
+    np.testing.assert_allclose(res.rows.train.log_cov, torch.log(cover).detach().numpy(), atol=1e-12)
+    assert np.array_equal(res.rows.train.count, chosen.sum(1))
+    np.testing.assert_allclose(res.d_hidden, h.grad.numpy(), atol=1e-12)
+    np.testing.assert_allclose(res.d_w, w.grad.numpy(), atol=1e-12)
+    assert (res.rows.grad[~chosen] == 0).all() and (res.d_hidden[4] == 0).all()
 
 
 def test_sequence_level_ratio_is_the_product_of_token_ratios_and_veto_rule():

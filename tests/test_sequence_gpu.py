@@ -44,6 +44,38 @@ def test_sequences_of_a_forward_pass():
     assert want.veto.sum() >= 1 and (want.veto == 0).sum() >= 1
 
 
+def test_coverage_minimum_and_mean_per_sequence():
+    """Z_min and mean Z over each sequence (Def. 5.2; Prop. 5.5's bound uses Z_min) from the
+    per-token ln Z of a forward pass, against the oracle's ln Z and its coverage statistics."""
+    w = inputs.WORKLOADS["c2_bf16_fwdbwd"]
+    batch = inputs.make_rows(w, seed=6, device=DEV, T=3000, V=8192)
+    batch.ids[7] = -1                                  # a state without a sampled token still counts
+    res = binding.dvp_forward(batch.train, batch.ids, 1e-3, infer_logits=batch.infer)
+    off = torch.tensor([0, 0, 1, 700, 3000, 3000], device=DEV)
+    got = binding.dvp_sequence_aggregate(res.log_ratio, off, 1e-4, log_cov=res.train.log_cov)
+    torch.cuda.synchronize()
+    import parity
+    want_rows = parity.run_oracle(batch.train, batch.infer, batch.ids, 1e-3)
+    lo, mean = oracle.dvp_coverage(want_rows.train.log_cov, off.cpu().numpy())
+    g_lo, g_mean = got.min_cov.cpu().numpy().astype(np.float64), got.mean_cov.cpu().numpy().astype(np.float64)
+    assert np.isposinf(g_lo[[0, 4]]).all() and np.isnan(g_mean[[0, 4]]).all()
+    np.testing.assert_allclose(g_lo[1:4], lo[1:4], atol=1e-4, rtol=0)
+    np.testing.assert_allclose(g_mean[1:4], mean[1:4], atol=1e-4, rtol=0)
+    assert (g_lo[1:4] <= g_mean[1:4] + 1e-7).all() and (g_mean[1:4] <= 1.0).all() and g_lo[3] < 1.0
+    # the other outputs do not change when the coverage is asked for
+    plain = binding.dvp_sequence_aggregate(res.log_ratio, off, 1e-4)
+    assert torch.equal(plain.veto, got.veto) and torch.equal(plain.n_valid, got.n_valid)
+    with pytest.raises(binding.DvpError):              # coverage outputs without the input
+        a = binding.SequenceArgs()
+        import ctypes
+        a.struct_size = ctypes.sizeof(binding.SequenceArgs)
+        a.T, a.S = 8, 1
+        a.seq_offsets, a.log_ratio, a.min_cov = off.data_ptr(), res.log_ratio.data_ptr(), got.min_cov.data_ptr()
+        st = binding.load_library().dvp_sequence_aggregate(ctypes.byref(a))
+        if st != binding.DVP_OK:
+            raise binding.DvpError(st, "dvp_sequence_aggregate")
+
+
 def test_special_values_empty_and_long_sequences():
     T = 40000
     g = torch.Generator().manual_seed(2)

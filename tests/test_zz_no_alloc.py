@@ -60,6 +60,8 @@ def test_static_workspace_variant_matches_the_ordinary_entry_point_twice():
             batch.hidden, batch.w_vocab, batch.ids, rho, batch.upstream, infer_logits=batch.infer)
         torch.cuda.synchronize()
         assert plain.workspace[:4].view(torch.int32).item() == 0
+        # the built-in array's own status word: no tensor-core kernel gave up waiting
+        assert binding.dvp_static_workspace_status() == 0
         _same(static, plain)
 
 
