@@ -8,10 +8,13 @@ the gradient (Def. 5.1, Def. 5.2, Prop. 5.4) for every token of the batch.
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--rho R]
   python bench.py --impl reference ...     # the fp64 CPU checker on host cores
 
-With N > 1 (launched by torchrun, one rank per GPU) every rank processes its
-own batch of the same shape: rows are independent, so there is no data-path
-collective, only the barrier and the max-over-ranks of the device time.
-Rank 0 prints one JSON line.
+With N > 1 every rank (one per GPU) processes its own batch of the same shape:
+rows are independent, so there is no data-path collective, only the barrier and
+the max-over-ranks of the device time.  Started without a launcher, ``--gpus N``
+starts the N ranks itself through ``torch.distributed.run`` on 127.0.0.1.
+Rank 0 prints one JSON line.  At N = 1 the default run appends, after the
+headline workload has freed its batch, one sub-object per other configuration
+(``c1_bf16_fwd``, ``c3_f32_heavy``, ``c4_fused_lmhead``), each timed the same way.
 """
 from __future__ import annotations
 
@@ -76,7 +79,7 @@ class ClockSampler:
             self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=self.file, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -169,9 +172,14 @@ def cpu_baseline(batch, rho, backward):
         rows += slab
         if total_t * used > 20.0:
             break
+    # the same checker on one thread, on fewer rows
+    one_rows = min(64, batch.train.shape[0])
+    one_t, _ = _oracle_sample(_host_rows(batch, 0, one_rows), rho, 1, backward)
     return {"value": rows / total_t, "unit": UNIT, "cores": used, "kind": "oracle",
             "sample": f"first {rows} rows of the batch (V={batch.train.shape[1]}), fp64, {used} threads, "
-                      f"rows split statically, {total_t:.2f} s wall"}
+                      f"rows split statically, {total_t:.2f} s wall",
+            "one_thread": {"value": one_rows / one_t, "unit": UNIT, "cores": 1,
+                           "sample": f"first {one_rows} rows, {one_t:.2f} s wall"}}
 
 
 def run_reference(args):
@@ -381,19 +389,98 @@ def run_ours(args):
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(batch, rho, w.backward)
+        if world == 1 and args.workload == "c2_bf16_fwdbwd" and not args.rows and not args.no_extras:
+            # the other configurations, one after the other, each with the device to itself
+            del batch, res, h_train, h_infer, d_train, d_infer, d_grad
+            if other is not None:
+                del res2
+            torch.cuda.empty_cache()
+            steps = max(3, min(args.steps, 10))
+            for name in ("c1_bf16_fwd", "c3_f32_heavy"):
+                line[name] = rows_extra(name, steps, dev, peak, peak_kind, args.no_cpu_baseline)
+                torch.cuda.empty_cache()
+            fargs = argparse.Namespace(**vars(args))
+            fargs.workload, fargs.rho, fargs.steps, fargs.e2e_steps = "c4_fused_lmhead", None, steps, 1
+            fline = fused_measure(fargs, 0, 1, dev)
+            line["c4_fused_lmhead"] = {k: fline[k] for k in ("ms_per_step", "value", "unit", "config", "clocks", "e2e",
+                                                             "roofline", "parity_sample", "cpu_baseline",
+                                                             "gpu_launches") if k in fline}
+            line["gpu_launches"] += sum(line[n].get("gpu_launches", 0)
+                                        for n in ("c1_bf16_fwd", "c3_f32_heavy", "c4_fused_lmhead"))
         print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()
 
 
+def rows_extra(name, steps, dev, peak, peak_kind, no_cpu_baseline):
+    """One row configuration beside the headline: ms per step, tokens/s, algorithmic GB/s and
+    its fraction of the peak, per threshold, with its own clock samples."""
+    import torch
+    from paper_2512_23087_b200 import binding, inputs
+    w = inputs.WORKLOADS[name]
+    batch = inputs.make_rows(w, seed=0, device=dev, T=w.T)
+    T, V = batch.train.shape
+    elem = batch.train.element_size()
+    grad_dtype = inputs.torch_dtype(w.grad_dtype or w.dtype)
+    alg_bytes = (2 * elem + (torch.empty(0, dtype=grad_dtype).element_size() if w.backward else 0)) * T * V
+    stream = torch.cuda.current_stream()
+    out = {"config": {"workload": name, "T": T, "V": V, "logits_dtype": w.dtype, "backward": w.backward,
+                      "l2": "inputs larger than L2, no flush"}, "bytes_per_launch": alg_bytes, "thresholds": []}
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    launches = 0
+    res = None
+    for rho in w.rhos:
+        for _ in range(3):
+            res = binding.dvp_forward(batch.train, batch.ids, rho, infer_logits=batch.infer,
+                                      upstream=batch.upstream if w.backward else None, grad_dtype=grad_dtype,
+                                      stream=stream, out=res)
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for _ in range(steps):
+            binding.dvp_forward(batch.train, batch.ids, rho, infer_logits=batch.infer,
+                                upstream=batch.upstream if w.backward else None, grad_dtype=grad_dtype,
+                                stream=stream, out=res)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        sec = ev0.elapsed_time(ev1) * 1e-3 / steps
+        launches += steps
+        out["thresholds"].append({"rho": rho, "ms_per_step": sec * 1e3, "value": T / sec, "unit": UNIT,
+                                  "achieved_gbs": alg_bytes / sec / 1e9, "frac": alg_bytes / sec / 1e9 / peak,
+                                  "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": alg_bytes / sec / 1e9 / 8000.0})
+    out["clocks"] = sampler.stop()
+    out["steps"] = steps
+    out["gpu_launches"] = launches
+    if not no_cpu_baseline:
+        cores = os.cpu_count() or 1
+        rows = 256
+        dt, used = _oracle_sample(_host_rows(batch, 0, rows), w.rhos[0], cores, w.backward)
+        one_t, _ = _oracle_sample(_host_rows(batch, 0, 32), w.rhos[0], 1, w.backward)
+        out["cpu_baseline"] = {"value": rows / dt, "unit": UNIT, "cores": used, "kind": "oracle",
+                               "sample": f"first {rows} rows, fp64, {used} threads, {dt:.2f} s wall",
+                               "one_thread": {"value": 32 / one_t, "unit": UNIT, "cores": 1,
+                                              "sample": f"first 32 rows, {one_t:.2f} s wall"}}
+    return out
+
+
 def run_fused(args):
     """Secondary line: the fused LM-head entry point (tensor-core bound)."""
+    import torch
+    rank, world, local = _dist_setup()
+    line = fused_measure(args, rank, world, torch.device("cuda", local))
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def fused_measure(args, rank, world, dev):
     import numpy as np
     import torch
     from paper_2512_23087_b200 import binding, inputs
 
-    rank, world, local = _dist_setup()
-    dev = torch.device("cuda", local)
+    local = dev.index or 0
     w = inputs.WORKLOADS[args.workload]
     rho = args.rho if args.rho is not None else w.rhos[0]
     T = args.rows if args.rows else w.T
@@ -472,11 +559,12 @@ def run_fused(args):
     tokens = T * world
     sec = ms * 1e-3 / args.steps
     flops = 2.0 * T * V * H + 4.0 * H * safe_total       # logits, then dH and dW over the safe entries
-    peak, kind = 1400.0, "fallback"
+    peak, burst, kind = 1400.0, 1590.0, "fallback"
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         try:
-            peak, kind = float(json.load(open(path))["bf16_tflops_sustained"]), "measured (sustained)"
+            pk = json.load(open(path))
+            peak, burst, kind = float(pk["bf16_tflops_sustained"]), float(pk["bf16_tflops"]), "measured (sustained)"
         except Exception:
             pass
     achieved = flops / sec / 1e12
@@ -496,23 +584,75 @@ def run_fused(args):
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "traffic": None, "peak_kind": f"of {kind}",
                      "kernel": "gemm_tn_kernel (three contractions per panel)",
-                     "flops_per_step": flops, "frac_of_nominal_2250": achieved / 2250.0},
+                     "flops_per_step": flops, "frac_of_burst": achieved / burst,
+                     "frac_of_nominal_2250": achieved / 2250.0},
     }
-    if rank == 0:
-        if world == 1 and not args.no_cpu_baseline:
-            import oracle
-            n = 16
-            bits = lambda x: x.detach().cpu().view(torch.int16).numpy().view(np.uint16)
-            t0 = time.perf_counter()
-            oracle.dvp_fused_lmhead(bits(batch.hidden[:n]), bits(batch.w_vocab), bits(batch.infer[:n]),
-                                    batch.ids[:n].cpu().numpy(), rho, batch.upstream[:n].cpu().numpy().astype("f8"))
-            dt = time.perf_counter() - t0
-            line["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
-                                    "sample": f"first {n} rows, full V and H, fp64 (numpy matmul threads + "
-                                              f"row oracle), {dt:.1f} s wall"}
-        print(json.dumps(line))
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        n = 16
+        bits = lambda x: x.detach().cpu().view(torch.int16).numpy().view(np.uint16)
+        t0 = time.perf_counter()
+        want = oracle.dvp_fused_lmhead(bits(batch.hidden[:n]), bits(batch.w_vocab), bits(batch.infer[:n]),
+                                       batch.ids[:n].cpu().numpy(), rho, batch.upstream[:n].cpu().numpy().astype("f8"))
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": f"first {n} rows, full V and H, fp64 (numpy matmul threads + "
+                                          f"row oracle), {dt:.1f} s wall"}
+        # the timed result's first rows against what the checker just computed: tokens whose
+        # safe-set size agrees (no logit flipped within rounding distance of the threshold)
+        # must match in log-probability (1e-4) and in their d_hidden row (1e-3 relative L2)
+        same = res.train.count[:n].cpu().numpy() == want.rows.train.count
+        lp = res.train.logp_mp[:n].cpu().double().numpy()
+        fin = np.isfinite(want.rows.train.logp_mp) & np.isfinite(lp) & same
+        lp_err = float(np.abs(lp - want.rows.train.logp_mp)[fin].max()) if fin.any() else 0.0
+        dh = res.d_hidden[:n].cpu().double().numpy()
+        num = np.linalg.norm(dh - want.d_hidden, axis=1)[same]
+        den = np.linalg.norm(want.d_hidden, axis=1)[same]
+        dh_err = float((num / np.maximum(den, 1e-6 * max(den.max(), 1e-300))).max()) if same.any() else 0.0
+        line["parity_sample"] = {"rows": n, "rows_with_the_same_safe_set_size": int(same.sum()),
+                                 "logp_mp_max_err": lp_err, "d_hidden_worst_row_rel_l2": dh_err,
+                                 "status_word": status}
+        if status != 0 or lp_err > 1e-4 or dh_err > 1e-3 or not same.any():
+            print(json.dumps(line))
+            raise SystemExit("fused LM-head result disagrees with the fp64 checker on its first rows")
+    return line
+
+
+def spawn_ranks(n: int) -> int:
+    """`bench.py --gpus N` without a launcher: start N ranks of this same command line, one per
+    GPU, through torch.distributed.run on the loopback address."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "WARN")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.call(cmd, env=env)
+
+
+def dry_run_ranks(args):
+    """The multi-rank plumbing without a GPU: rendezvous over gloo, shard the rows, take the
+    maximum of a per-rank number the way the timed paths do, rank 0 prints one line."""
+    import torch
+    import torch.distributed as dist
+    from paper_2512_23087_b200 import inputs
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
     if world > 1:
-        torch.distributed.destroy_process_group()
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("gloo")
+    w = inputs.WORKLOADS[args.workload]
+    r0, r1 = inputs.shard_rows(w.T * world, rank, world)     # weak scaling: every rank its own w.T rows
+    t = torch.tensor([float(rank + 1), float(r1 - r0)], dtype=torch.float64)
+    if world > 1:
+        dist.barrier()
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "n_gpus": world, "max_over_ranks": t[0].item(),
+                          "rows_per_rank": int(t[1].item()), "scaling": "weak"}))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 def main():
@@ -528,7 +668,14 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--panel-rows", type=int, default=0, help="fused workload: tokens per panel")
+    ap.add_argument("--no-extras", action="store_true", help="headline workload only")
+    ap.add_argument("--dry-run-ranks", action="store_true",
+                    help="ranks only rendezvous (gloo, no GPU) and reduce a number: checks the launch path")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus))
+    if args.dry_run_ranks:
+        return dry_run_ranks(args)
     if args.workload == "c4_fused_lmhead":
         if args.impl == "reference":
             if int(os.environ.get("RANK", "0")) == 0:

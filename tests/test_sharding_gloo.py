@@ -70,3 +70,21 @@ def test_two_gloo_ranks_reproduce_the_single_rank_result(tmp_path):
     assert np.array_equal(rows[:, 1], want.log_ratio)
     assert np.array_equal(rows[:, 2], want.train.count.astype(np.float64))
     assert got["t_max"] == 10.0 + world - 1
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`bench.py --gpus 2` started plainly: it must launch two ranks itself (torch.distributed.run
+    on 127.0.0.1), which here only rendezvous over gloo, shard the rows and reduce a number."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--dry-run-ranks"],
+                         capture_output=True, text=True, env=env, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                   # rank 0 alone prints
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["max_over_ranks"] == 2.0 and line["scaling"] == "weak"
+    assert line["rows_per_rank"] == inputs.WORKLOADS["c2_bf16_fwdbwd"].T
