@@ -283,6 +283,20 @@ __device__ __forceinline__ SumCount block_reduce_sumcount(SumCount v, float *scr
   return r;
 }
 
+// Maximum over the block.  scratch: 32 floats.  Result valid in every thread.
+__device__ __forceinline__ float block_reduce_max(float v, float *scratch) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  __syncthreads();
+  if (lane == 0) scratch[warp] = v;
+  __syncthreads();
+  float r = lane < nwarp ? scratch[lane] : kNegInf;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) r = fmaxf(r, __shfl_xor_sync(0xffffffffu, r, o));
+  return r;
+}
+
 // ---- per-row bookkeeping shared by all row kernels ---------------------------
 
 struct RowParams {
@@ -305,6 +319,12 @@ struct RowParams {
   // ln pi^mp_infer(a) per token, and flags whose DVP_FLAG_IN_TRAIN bit says "a in V'_S"
   const float *given_logp_mp_i;
   const uint8_t *given_flags_i;
+  // 4-byte logits whose row maxima an earlier launch left, in pieces: the maximum of row t is the
+  // largest of given_max[t * given_max_ld + i], i < given_max_n.  The vectorised kernel then needs
+  // one sweep less; the other kernels ignore it.
+  const float *given_max;
+  long long given_max_ld;
+  int given_max_n;
 };
 
 __device__ __forceinline__ long long load_id(const void *ids, int is_i32, long long t) {

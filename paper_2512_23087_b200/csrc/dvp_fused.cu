@@ -128,7 +128,8 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct FusedLayout {
   long long Vp, Tp, panel;
-  size_t off_scalars, off_lpt, off_lpi, off_fli, off_flt, off_wt, off_ht, off_z, off_g, total;
+  size_t off_scalars, off_lpt, off_lpi, off_fli, off_flt, off_wt, off_ht, off_z, off_g, off_rmax, total;
+  long long max_pieces;
 };
 
 bool fused_layout(const dvp_fused_args *a, FusedLayout *L) {
@@ -159,6 +160,8 @@ bool fused_layout(const dvp_fused_args *a, FusedLayout *L) {
   L->off_ht = take((size_t)a->H * L->Tp * 2);
   L->off_z = take((size_t)panel * L->Vp * 4);
   L->off_g = take((size_t)panel * L->Vp * 2);
+  L->max_pieces = (a->V + gemm::kBN - 1) / gemm::kBN;  // one per tile column of the logits contraction
+  L->off_rmax = take((size_t)panel * L->max_pieces * 4);
   L->total = o;
   return true;
 }
@@ -256,6 +259,7 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
   __half *ht16 = reinterpret_cast<__half *>(ws + L.off_ht);   // [H, Tp]: hidden^T
   float *z = reinterpret_cast<float *>(ws + L.off_z);         // [panel, Vp] logits
   __half *g16 = reinterpret_cast<__half *>(ws + L.off_g);     // [panel, Vp] scaled gradient
+  float *rmax = reinterpret_cast<float *>(ws + L.off_rmax);   // [panel, max_pieces] row maxima of z in pieces
   const __nv_bfloat16 *hidden = static_cast<const __nv_bfloat16 *>(a->hidden);
   const __nv_bfloat16 *w = static_cast<const __nv_bfloat16 *>(a->w_vocab);
   const int T = (int)a->T, H = (int)a->H, V = (int)a->V;
@@ -290,8 +294,11 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
   for (long long r0 = 0; r0 < a->T; r0 += L.panel, ++panel_index) {
     const int rows = (int)((a->T - r0 < L.panel) ? a->T - r0 : L.panel);
     // logits of the panel: z = hidden[r0 : r0 + rows] x W^T (bf16 operands, fp32 accumulate)
+    // its epilogue also leaves each row's maximum, one piece per tile column: the row kernel
+    // then knows the threshold before it reads the panel and needs one sweep less
     cudaError_t e = gemm::launch_gemm_tn(hidden + r0 * a->ld_hidden, a->ld_hidden, w, a->ld_w, z, L.Vp,
-                                         rows, V, H, true, 1.f, nullptr, false, &sc->status, sms, s);
+                                         rows, V, H, true, 1.f, nullptr, false, &sc->status, sms, s, false,
+                                         false, 1, rmax, L.max_pieces);
     if (e != cudaSuccess) return e == cudaErrorInvalidValue ? DVP_ERR_UNSUPPORTED : DVP_ERR_CUDA;
     // rows of the panel: statistics and G = scale * dLoss/dz in float16
     RowParams p{};
@@ -306,6 +313,9 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
     p.ld_grad = L.Vp;
     p.log_rho = log_rho;
     p.id_is_i32 = a->id_dtype == DVP_ID_I32;
+    p.given_max = rmax;
+    p.given_max_ld = L.max_pieces;
+    p.given_max_n = (int)L.max_pieces;
     p.out_t = offset_side(a->train, r0, mask_words);
     p.out_t.logp_mp = lpt + r0;
     p.flags = flt + r0;

@@ -46,6 +46,8 @@ struct Params {
   int a_mn_major;          // A is stored transposed, [K, M] with M contiguous (pair kernel only)
   int split_k;             // pair kernel: each tile's K range is cut into this many units whose
                            // results are added to C with atomics (C zeroed or accumulated into)
+  float *row_max;          // optional (pair kernel, no split, no accumulation): row_max[row * row_max_ld + tn]
+  long long row_max_ld;    // = the maximum of row `row` of C over the columns of tile column tn
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -537,12 +539,18 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       tc_fence_after();
       const int row = tm * kPairBM + (int)rank * kBM + quarter * 32 + lane;
       float *crow = p.C + (long long)row * p.ldc;
+      float row_hi = -__builtin_huge_valf();  // maximum of what this thread stores of its row
 #pragma unroll 1
       for (int c0 = 0; c0 < kBN; c0 += 32) {
         uint32_t r[32];
         tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kBN + c0, r);
         tmem_wait_ld();
         const int col = tn * kBN + c0;
+        if (p.row_max && row < p.M) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (col + j < p.N) row_hi = fmaxf(row_hi, alpha * __uint_as_float(r[j]));
+        }
         if (row < p.M && col < p.N) {
           if (p.split_k > 1) {  // this unit holds a part of the sum: add it
             for (int j = 0; j < 32 && col + j < p.N; ++j) atomicAdd(crow + col + j, alpha * __uint_as_float(r[j]));
@@ -574,6 +582,7 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           }
         }
       }
+      if (p.row_max && row < p.M) p.row_max[(long long)row * p.row_max_ld + tn] = row_hi;
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_remote(map_to_rank(smem_u32(&sh->tmem_empty[buf]), 0));
@@ -637,14 +646,18 @@ inline cudaError_t launch_gemm_tn(const void *A, long long lda, const void *B, l
                                   long long ldc, int M, int N, int K, bool is_bf16, float alpha,
                                   const float *alpha_dev, bool accumulate, int *status, int sm_count,
                                   cudaStream_t stream, bool single_block_tiles = false,
-                                  bool a_mn_major = false, int split_k = 1) {
+                                  bool a_mn_major = false, int split_k = 1, float *row_max = nullptr,
+                                  long long row_max_ld = 0) {
   if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
   if (lda % 8 || ldb % 8 || ldc % 8 || (uintptr_t)A % 16 || (uintptr_t)B % 16 || (uintptr_t)C % 32)
     return cudaErrorInvalidValue;
   if (a_mn_major && single_block_tiles) return cudaErrorInvalidValue;
   // every K range of a split needs work; the split results meet in C by atomic adds
   if (single_block_tiles || split_k < 1 || (K + kBK - 1) / kBK < 2 * split_k) split_k = 1;
-  Params p{C, ldc, M, N, K, alpha, alpha_dev, accumulate ? 1 : 0, status, a_mn_major ? 1 : 0, split_k};
+  // per-tile row maxima are those of the stored values: only where a tile is stored once, whole
+  if (row_max && (single_block_tiles || split_k > 1 || accumulate)) return cudaErrorInvalidValue;
+  Params p{C, ldc, M, N, K, alpha, alpha_dev, accumulate ? 1 : 0, status, a_mn_major ? 1 : 0, split_k,
+           row_max, row_max_ld};
   if (split_k > 1 && !accumulate) {
     const cudaError_t z = cudaMemset2DAsync(C, (size_t)ldc * 4, 0, (size_t)N * 4, (size_t)M, stream);
     if (z != cudaSuccess) return z;
