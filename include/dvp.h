@@ -119,9 +119,9 @@ typedef struct {
                     /* (<= 0; 1 - Z is the total variation distance between    */
                     /* pi^mp and pi in the proof of Prop. 5.5).  Formed in     */
                     /* double from the two sums the kernel holds, not from the */
-                    /* float outputs lse_safe and lse; Z itself is good to a    */
-                    /* few 1e-6, so 1 - Z keeps 1e-3 relative accuracy down to  */
-                    /* about 1 - Z = 4e-3                                      */
+                    /* float outputs lse_safe and lse; Z itself is good to      */
+                    /* about 1e-5 (float32 sums), so 1 - Z keeps 1e-3 relative  */
+                    /* accuracy down to about 1 - Z = 1e-2                      */
 } dvp_side_out;
 
 /*
@@ -475,6 +475,21 @@ int dvp_gemm_tn(const void *a, int64_t lda, const void *b, int64_t ldb, float *c
  * DVP_ERR_CUDA.
  */
 int dvp_row_wait_status(uint32_t *status_out);
+
+/*
+ * dvp_debug_bounds_status -- the library can be built a second time with every
+ * shared-memory index of the row kernels' on-chip tables and every global element
+ * offset they form compared with its extent (python -m paper_2512_23087_b200.build
+ * --debug-bounds gives libdvp_b200_bounds.so).  In that build an index out of range
+ * is never used: the access is skipped and a code is OR-ed into a per-device word
+ * (1 granule-bound table, 2 hot list, 4 granule index, 8 global offset, 16 candidate
+ * ring, 32 candidate list, 64 resident slot).  This call waits for all work on the
+ * current device, copies the word to *status_out (a host pointer) and clears it; 0
+ * means that no check has failed since the last call.  The ordinary build has no
+ * checks and returns DVP_ERR_UNSUPPORTED.  The paper has no counterpart: it stands
+ * in for a memory checker.  Errors: DVP_ERR_INVALID_ARG (NULL), DVP_ERR_CUDA.
+ */
+int dvp_debug_bounds_status(uint32_t *status_out);
 
 /*
  * Bytes of device workspace the entry point needs for `args` (a pointer to

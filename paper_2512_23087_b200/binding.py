@@ -7,6 +7,7 @@ been built, the first call raises.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
 import os
 from types import SimpleNamespace
@@ -15,6 +16,7 @@ import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libdvp_b200.so")
+BOUNDS_LIB_PATH = os.path.join(_HERE, "libdvp_b200_bounds.so")   # the bounds-checking build
 
 DVP_OK, DVP_ERR_INVALID_ARG, DVP_ERR_UNSUPPORTED, DVP_ERR_WORKSPACE, DVP_ERR_CUDA = range(5)
 DVP_F32, DVP_BF16, DVP_F16 = 0, 1, 2
@@ -28,7 +30,7 @@ DVP_WEIGHT_NONE, DVP_WEIGHT_RATIO, DVP_WEIGHT_TRUNCATE, DVP_WEIGHT_MASK = 0, 1, 
 EXPORTS = ("dvp_forward", "dvp_backward", "dvp_fused_lmhead_forward_backward",
            "dvp_fused_lmhead_forward_backward_static", "dvp_sequence_aggregate", "dvp_monitor", "dvp_gemm_tn",
            "dvp_workspace_bytes", "dvp_status_string", "dvp_version", "dvp_row_wait_status",
-           "dvp_static_workspace_status")
+           "dvp_static_workspace_status", "dvp_debug_bounds_status")
 
 _DTYPES = {torch.float32: DVP_F32, torch.bfloat16: DVP_BF16, torch.float16: DVP_F16}
 _SIDE_FIELDS = ("max", "lse", "lse_safe", "logp", "logp_mp", "comp_mp", "count", "mask", "log_cov")
@@ -216,8 +218,39 @@ def load_library() -> ctypes.CDLL:
         lib.dvp_row_wait_status.restype = ctypes.c_int
         lib.dvp_static_workspace_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
         lib.dvp_static_workspace_status.restype = ctypes.c_int
+        lib.dvp_debug_bounds_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
+        lib.dvp_debug_bounds_status.restype = ctypes.c_int
         _lib = lib
     return _lib
+
+
+@contextlib.contextmanager
+def bounds_checking_library():
+    """Inside the block every call of this module goes to the bounds-checking build of the
+    library (``python -m paper_2512_23087_b200.build --debug-bounds``), whose kernels compare
+    every index of their on-chip tables and every global offset with its extent;
+    ``dvp_debug_bounds_status()`` then tells whether any check failed."""
+    global _lib, LIB_PATH
+    if not os.path.exists(BOUNDS_LIB_PATH):
+        raise RuntimeError(f"{BOUNDS_LIB_PATH} is missing: build it with "
+                           "`python -m paper_2512_23087_b200.build --debug-bounds`")
+    saved = (_lib, LIB_PATH)
+    _lib, LIB_PATH = None, BOUNDS_LIB_PATH
+    try:
+        yield load_library()
+    finally:
+        _lib, LIB_PATH = saved
+
+
+def dvp_debug_bounds_status() -> int:
+    """Waits for the current device and returns (and clears) the word into which the
+    bounds-checking build ORs a code for every index it found out of range; raises
+    ``DvpError(DVP_ERR_UNSUPPORTED)`` on the ordinary build, which has no checks."""
+    out = ctypes.c_uint32(0)
+    st = load_library().dvp_debug_bounds_status(ctypes.byref(out))
+    if st != DVP_OK:
+        raise DvpError(st, "dvp_debug_bounds_status")
+    return int(out.value)
 
 
 def status_string(status: int) -> str:

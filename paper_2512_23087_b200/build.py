@@ -2,7 +2,8 @@
 
 ``build()`` compiles every ``csrc/*.cu`` to an object file (in parallel) and
 links ``libdvp_b200.so`` beside this file.  Objects are rebuilt only when a
-source or header is newer.  Run as ``python -m paper_2512_23087_b200.build``.
+source or header is newer.  Run as ``python -m paper_2512_23087_b200.build``;
+``--debug-bounds`` builds the bounds-checking library instead.
 """
 from __future__ import annotations
 
@@ -37,20 +38,29 @@ def _newest_header() -> float:
     return max(os.path.getmtime(h) for h in hdrs)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    os.makedirs(OBJ, exist_ok=True)
+LIB_BOUNDS = os.path.join(HERE, "libdvp_b200_bounds.so")
+
+
+def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False) -> str:
+    """``debug_bounds``: the second library, compiled with -DDVP_DEBUG_BOUNDS (every index of
+    the row kernels' on-chip tables and every global offset checked, reported through
+    ``dvp_debug_bounds_status``), as ``libdvp_b200_bounds.so``."""
+    obj_dir = OBJ + ("_bounds" if debug_bounds else "")
+    lib = LIB_BOUNDS if debug_bounds else LIB
+    extra = ["-DDVP_DEBUG_BOUNDS"] if debug_bounds else []
+    os.makedirs(obj_dir, exist_ok=True)
     srcs = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
     hdr_time = _newest_header()
     nvcc = _nvcc()
     jobs = []
     objs = []
     for src in srcs:
-        obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         stale = force or not os.path.exists(obj) or \
             os.path.getmtime(obj) < max(os.path.getmtime(src), hdr_time)
         if stale:
-            cmd = [nvcc, *NVCC_FLAGS, "-c", src, "-o", obj]
+            cmd = [nvcc, *NVCC_FLAGS, *extra, "-c", src, "-o", obj]
             if verbose:
                 cmd.insert(1, "-Xptxas")
                 cmd.insert(2, "-v")
@@ -67,12 +77,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
             for log in ex.map(run, jobs):
                 if verbose and log:
                     print(log, file=sys.stderr)
-    if jobs or not os.path.exists(LIB):
-        tmp = LIB + f".{os.getpid()}.tmp"
+    if jobs or not os.path.exists(lib):
+        tmp = lib + f".{os.getpid()}.tmp"
         run([nvcc, "-shared", "-o", tmp, *objs, "-lcudart"])
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug_bounds="--debug-bounds" in sys.argv))

@@ -124,6 +124,16 @@ int dvp_row_wait_status(uint32_t *status_out) {
   return dvp::read_and_clear_row_status(status_out) == cudaSuccess ? DVP_OK : DVP_ERR_CUDA;
 }
 
+int dvp_debug_bounds_status(uint32_t *status_out) {
+  if (!status_out) return DVP_ERR_INVALID_ARG;
+#ifdef DVP_DEBUG_BOUNDS
+  return dvp::read_and_clear_bounds_status(status_out) == cudaSuccess ? DVP_OK : DVP_ERR_CUDA;
+#else
+  *status_out = 0;
+  return DVP_ERR_UNSUPPORTED;  // this library was built without the checks
+#endif
+}
+
 const char *dvp_status_string(int status) {
   switch (status) {
     case DVP_OK: return "DVP_OK";

@@ -20,6 +20,57 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// ---- bounds-checking build (-DDVP_DEBUG_BOUNDS) ------------------------------------
+// Stands in for a memory checker: every shared-memory index of the row kernels' tables
+// (granule bounds, hot lists, candidate rings and lists, resident slots) and every global
+// element offset they form is compared with its extent.  An index out of range is not
+// used: the access is skipped and a code is OR-ed into a per-device status word that
+// dvp_debug_bounds_status reads.  Nothing traps.  In the ordinary build the checks
+// compile to nothing.
+enum : unsigned {
+  DVP_OOB_BOUND = 1,    // granule-bound table
+  DVP_OOB_HOT = 2,      // hot-list entry
+  DVP_OOB_GRANULE = 4,  // granule index outside the row
+  DVP_OOB_GLOBAL = 8,   // global element offset outside the row
+  DVP_OOB_RING = 16,    // candidate ring slot
+  DVP_OOB_LIST = 32,    // candidate list entry
+  DVP_OOB_SLOT = 64     // resident-row slot or its bytes
+};
+#ifdef DVP_DEBUG_BOUNDS
+struct BoundsCtx {
+  unsigned int *status;
+  long long n_bound, n_hot, n_gran, V, n_ring, n_list, n_slot;
+};
+// one instance per block (a __shared__ variable of a device function)
+__device__ __forceinline__ BoundsCtx &bounds_ctx() {
+  __shared__ BoundsCtx c;
+  return c;
+}
+__device__ __forceinline__ bool bounds_ok(long long i, long long n, unsigned code) {
+  if (i >= 0 && i < n) return true;
+  if (bounds_ctx().status) atomicOr(bounds_ctx().status, code);
+  return false;
+}
+#define DVP_IN(i, field, code) ::dvp::bounds_ok((long long)(i), ::dvp::bounds_ctx().field, code)
+#define DVP_BOUNDS_SET(field, value) \
+  do { if (threadIdx.x == 0) ::dvp::bounds_ctx().field = (value); } while (0)
+#define DVP_BOUNDS_BEGIN(ptr)                                                                    \
+  do {                                                                                           \
+    if (threadIdx.x == 0) {                                                                      \
+      ::dvp::BoundsCtx &c_ = ::dvp::bounds_ctx();                                                \
+      c_.status = (ptr);                                                                         \
+      c_.n_bound = c_.n_hot = c_.n_gran = c_.V = c_.n_ring = c_.n_list = c_.n_slot = 0;                     \
+    }                                                                                            \
+    __syncthreads();                                                                             \
+  } while (0)
+#define DVP_BOUNDS_SYNC() __syncthreads()
+#else
+#define DVP_IN(i, field, code) true
+#define DVP_BOUNDS_SET(field, value) do { } while (0)
+#define DVP_BOUNDS_BEGIN(ptr) do { } while (0)
+#define DVP_BOUNDS_SYNC() do { } while (0)
+#endif
+
 // 16-byte read-only load that does not allocate in L1: each logit is consumed
 // once per sweep, re-reads are served by L2.
 __device__ __forceinline__ uint4 ld_stream16(const void *p) {
@@ -325,6 +376,7 @@ struct RowParams {
   const float *given_max;
   long long given_max_ld;
   int given_max_n;
+  unsigned int *bounds_status;  // the bounds-checking build's status word; unused otherwise
 };
 
 __device__ __forceinline__ long long load_id(const void *ids, int is_i32, long long t) {
@@ -468,6 +520,7 @@ struct BackwardParams {
   int id_is_i32;
   int mode;
   float mask_value;
+  unsigned int *bounds_status;  // the bounds-checking build's status word; unused otherwise
 };
 
 // Launchers (dvp_rows.cu).  `hint`: threads per block in the low 16 bits,
@@ -479,5 +532,10 @@ cudaError_t launch_backward_kernel(const BackwardParams &p, int logits_dtype, in
 
 // Synchronises the current device, reads the resident-row kernel's status word and clears it.
 cudaError_t read_and_clear_row_status(uint32_t *host_out);
+
+// Device address of the bounds-checking build's status word (nullptr in the ordinary build),
+// and its value after a device synchronisation (cleared by the read).
+unsigned int *bounds_status_word();
+cudaError_t read_and_clear_bounds_status(uint32_t *host_out);
 
 }  // namespace dvp

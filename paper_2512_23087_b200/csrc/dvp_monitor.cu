@@ -95,6 +95,7 @@ struct MonitorParams {
   const void *train, *infer;
   long long T, V, ld_train, ld_infer;
   float *kl_it, *kl_ti, *h_t, *h_i;
+  unsigned int *bounds_status;  // the bounds-checking build's status word; unused otherwise
 };
 
 __device__ __forceinline__ void monitor_finish(const MonitorParams &p, long long t, const Moments &a,
@@ -119,6 +120,10 @@ __global__ void __launch_bounds__(256, 3) dvp_monitor_kernel(const MonitorParams
   const TIn *zt = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
   const TIn *zi = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
   const int V = (int)p.V;
+  DVP_BOUNDS_BEGIN(p.bounds_status);
+  DVP_BOUNDS_SET(n_gran, (V + kElems - 1) / kElems);
+  DVP_BOUNDS_SET(V, V);
+  DVP_BOUNDS_SYNC();
   Moments a = {kNegInf, kNegInf, 0.f, 0.f, 0.f}, b = a;
   if constexpr (kVector) {
     const int n_full = V / kElems, n_gran = (V + kElems - 1) / kElems;
@@ -202,7 +207,8 @@ extern "C" int dvp_monitor(const dvp_monitor_args *a) {
   if (!a->train_logits || !a->infer_logits || a->ld_train < a->V || a->ld_infer < a->V)
     return DVP_ERR_INVALID_ARG;
   dvp::MonitorParams p{a->train_logits, a->infer_logits, a->T, a->V, a->ld_train, a->ld_infer,
-                       a->kl_infer_train, a->kl_train_infer, a->entropy_train, a->entropy_infer};
+                       a->kl_infer_train, a->kl_train_infer, a->entropy_train, a->entropy_infer,
+                       dvp::bounds_status_word()};
   cudaStream_t s = static_cast<cudaStream_t>(a->stream);
   cudaError_t e;
   switch (a->logits_dtype) {

@@ -39,6 +39,22 @@ struct Granule {
 
   // Granule `g` of a row of V elements; elements past V read as -inf.
   __device__ __forceinline__ void load_any(const TIn *row, int V, int n_full, int g) {
+    // granules past the end of the row are legal here (they read as -inf); what the
+    // bounds-checking build verifies is that the vector load below stays inside the row
+    if (g < 0 || (g < n_full && !DVP_IN((long long)g * kElems + kElems - 1, V, DVP_OOB_GLOBAL))) {
+      DVP_IN(g, n_gran, DVP_OOB_GRANULE);
+      const TIn fill = Storage<TIn>::narrow(kNegInf);
+      uint32_t f = 0;
+      if constexpr (sizeof(TIn) == 4) {
+        f = *reinterpret_cast<const uint32_t *>(&fill);
+      } else {
+        const uint32_t h = *reinterpret_cast<const uint16_t *>(&fill);
+        f = h | (h << 16);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) w[i] = f;
+      return;
+    }
     if (g < n_full) {
       load(row + (size_t)g * kElems);
     } else {
@@ -178,7 +194,8 @@ __device__ __forceinline__ HotList build_hot_list(const uint16_t *bound, int n_s
     uint32_t acc = 0;  // bit s: first granule of step step0 + s, bit 16 + s: second granule
     const int n = min(16, n_steps - step0);
     for (int s = 0; s < n; ++s) {
-      const uint32_t w = words[(step0 + s) * blockDim.x + tid];
+      const int wi = (step0 + s) * (int)blockDim.x + tid;
+      const uint32_t w = DVP_IN(2 * wi + 1, n_bound, DVP_OOB_BOUND) ? words[wi] : 0u;
       const uint32_t m = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&w), tau2);
       acc |= (m & 0x00010001u) << s;
     }
@@ -235,7 +252,14 @@ __device__ __forceinline__ void granule_grad(const Granule<TIn> &gr, TGrad *grow
     out[j] = x[j] >= tau ? coef * ex2((x[j] - m) * kLog2e) : 0.f;
     if (j == ja) out[j] = g_a;
   }
+  // a granule past the end of the row is legal here (a hot list built for a threshold of -inf
+  // names them): nothing of it is stored below.  A negative index is not.
+  if (g < 0) {
+    DVP_IN(g, n_gran, DVP_OOB_GRANULE);
+    return;
+  }
   if (g < n_full) {
+    if (!DVP_IN((long long)g * kElems + kElems - 1, V, DVP_OOB_GLOBAL)) return;
     store_granule<TGrad, kElems>(grow + (size_t)g * kElems, out);
   } else {
 #pragma unroll
@@ -252,7 +276,8 @@ struct Stage {
   Granule<TIn> g[kStage];
   __device__ __forceinline__ void load(const TIn *row, int V, int n_full, int step) {
     const int g0 = step * kStage * (int)blockDim.x + threadIdx.x;
-    if ((step + 1) * kStage * (int)blockDim.x <= n_full) {
+    if ((step + 1) * kStage * (int)blockDim.x <= n_full &&
+        DVP_IN(g0 + (kStage - 1) * (int)blockDim.x, n_gran, DVP_OOB_GRANULE)) {
 #pragma unroll
       for (int u = 0; u < kStage; ++u)
         g[u].load(row + (size_t)(g0 + u * (int)blockDim.x) * Granule<TIn>::kElems);
@@ -271,7 +296,8 @@ __device__ __forceinline__ void absorb_stage(const Stage<TIn, kStage> &st, int s
 #pragma unroll
   for (int u = 0; u < kStage; ++u) {
     const float gm = st.g[u].max();
-    bound[bound_index<kStage>(step * kStage + u, threadIdx.x)] = bf16_bits_round_up(gm);
+    const int bi = bound_index<kStage>(step * kStage + u, threadIdx.x);
+    if (DVP_IN(bi, n_bound, DVP_OOB_BOUND)) bound[bi] = bf16_bits_round_up(gm);
     cm = fmaxf(cm, gm);
   }
   if (cm > kNegInf) {
@@ -399,8 +425,9 @@ __device__ __forceinline__ SumCount row_sweep2(const TIn *row, int V, int a, flo
   if (hot.fits()) {
     const int wbase = tid & ~31, lane = tid & 31;
     for (int q = lane; q < hot.count; q += 64) {
+      if (!DVP_IN(q, n_hot, DVP_OOB_HOT)) break;
       const uint32_t e0 = hot.slots[q];
-      const bool two = q + 32 < hot.count;
+      const bool two = q + 32 < hot.count && DVP_IN(q + 32, n_hot, DVP_OOB_HOT);
       const uint32_t e1 = two ? hot.slots[q + 32] : e0;
       const int g0 = (int)(e0 >> 5) * (int)blockDim.x + wbase + (int)(e0 & 31);
       const int g1 = (int)(e1 >> 5) * (int)blockDim.x + wbase + (int)(e1 & 31);
@@ -412,6 +439,7 @@ __device__ __forceinline__ SumCount row_sweep2(const TIn *row, int V, int a, flo
     }
   } else {
     for (int i = 0; i < n_slots; ++i) {
+      if (!DVP_IN(bound_index<kStage>(i, tid), n_bound, DVP_OOB_BOUND)) break;
       if (bf16_bits_to_float(bound[bound_index<kStage>(i, tid)]) >= tau_b) {
         const int g = i * (int)blockDim.x + tid;
         Granule<TIn> gr;
@@ -433,7 +461,8 @@ __device__ __forceinline__ void absorb_given(const Granule<TIn> &gr, int slot, i
                                              GivenSums &acc, uint16_t *bound) {
   constexpr int kElems = Granule<TIn>::kElems;
   const int g = slot * (int)blockDim.x + (int)threadIdx.x;
-  bound[bound_index<kStage>(slot, threadIdx.x)] = bf16_bits_round_up(gr.max());
+  const int bi = bound_index<kStage>(slot, threadIdx.x);
+  if (DVP_IN(bi, n_bound, DVP_OOB_BOUND)) bound[bi] = bf16_bits_round_up(gr.max());
   float x[kElems];
   gr.get(x);
   const int ja = a - g * kElems;
@@ -594,6 +623,7 @@ __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int
   for (int i = 0; i < n_slots; ++i) {
     const int gi = i * (int)blockDim.x + tid;
     if (gi >= n_gran) break;
+    if (!DVP_IN(bound_index<kStage>(i, tid), n_bound, DVP_OOB_BOUND)) break;
     if (bf16_bits_to_float(bound[bound_index<kStage>(i, tid)]) >= tau_b) {
       if (!listed) {
         Granule<TIn> gr;
@@ -601,7 +631,8 @@ __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int
         granule_grad<TIn, TGrad>(gr, grow, V, n_full, gi, a_live, tau, st.m, coef, g_a);
       }
     } else if (gi < n_full) {
-      store_zero_granule<TGrad, kElems>(grow + (size_t)gi * kElems);
+      if (DVP_IN((long long)gi * kElems + kElems - 1, V, DVP_OOB_GLOBAL))
+        store_zero_granule<TGrad, kElems>(grow + (size_t)gi * kElems);
     } else {
       for (int j = 0; j < kElems; ++j) {
         const long long k = (long long)gi * kElems + j;
@@ -612,8 +643,9 @@ __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int
   if (listed) {
     const int wbase = tid & ~31, lane = tid & 31;
     for (int q = lane; q < hot.count; q += 64) {
+      if (!DVP_IN(q, n_hot, DVP_OOB_HOT)) break;
       const uint32_t e0 = hot.slots[q];
-      const bool two = q + 32 < hot.count;
+      const bool two = q + 32 < hot.count && DVP_IN(q + 32, n_hot, DVP_OOB_HOT);
       const uint32_t e1 = two ? hot.slots[q + 32] : e0;
       const int g0 = (int)(e0 >> 5) * (int)blockDim.x + wbase + (int)(e0 & 31);
       const int g1 = (int)(e1 >> 5) * (int)blockDim.x + wbase + (int)(e1 & 31);
@@ -646,6 +678,7 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
   uint16_t *bound = reinterpret_cast<uint16_t *>(smem + smem_words_fixed(blockDim.x));
 
   constexpr int kElems = Granule<TIn>::kElems;
+  DVP_BOUNDS_BEGIN(p.bounds_status);
   const long long t = blockIdx.x / kCluster;
   const int rank = kCluster > 1 ? (int)cluster_rank() : 0;
   const long long id = p.ids ? load_id(p.ids, p.id_is_i32, t) : -1;
@@ -657,6 +690,16 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
   const int per_rank = (n_gran + kCluster - 1) / kCluster;
   const int off = min(rank * per_rank, n_gran) * kElems;
   const int v_part = max(0, min(V - off, per_rank * kElems));
+#ifdef DVP_DEBUG_BOUNDS
+  {  // extents of this block's part of the row and of its tables
+    const int part_gran = (v_part + kElems - 1) / kElems, per_step = kStage * (int)blockDim.x;
+    DVP_BOUNDS_SET(n_gran, part_gran);
+    DVP_BOUNDS_SET(V, v_part);
+    DVP_BOUNDS_SET(n_bound, (long long)((part_gran + per_step - 1) / per_step) * per_step);
+    DVP_BOUNDS_SET(n_hot, kHotCap);  // entries of one warp's hot list
+    DVP_BOUNDS_SYNC();
+  }
+#endif
 
   const TIn *trow = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
   uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * ((p.V + 31) / 32) : nullptr;
@@ -824,6 +867,10 @@ __global__ void dvp_row_kernel_scalar(const RowParams p) {
 template <typename TIn, typename TGrad, int kStage, bool kVector>
 __global__ void dvp_backward_kernel(const BackwardParams p) {
   const long long t = blockIdx.x;
+  DVP_BOUNDS_BEGIN(p.bounds_status);
+  DVP_BOUNDS_SET(n_gran, (p.V + Granule<TIn>::kElems - 1) / Granule<TIn>::kElems);
+  DVP_BOUNDS_SET(V, p.V);
+  DVP_BOUNDS_SYNC();
   const TIn *row = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
   TGrad *grow = reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad;
   const long long id = load_id(p.ids, p.id_is_i32, t);

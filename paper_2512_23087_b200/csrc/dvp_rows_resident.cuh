@@ -329,7 +329,10 @@ struct Walk {
   Cursor res, str;  // next use of the resident and of the stream ring
   Waiter w;
 
-  __device__ __forceinline__ uint32_t slot_addr(int slot) const { return base + (uint32_t)slot * kSlotBytes; }
+  __device__ __forceinline__ uint32_t slot_addr(int slot) const {
+    if (!DVP_IN(slot, n_slot, DVP_OOB_SLOT)) slot = 0;  // bounds-checking build: reported, slot 0 read instead
+    return base + (uint32_t)slot * kSlotBytes;
+  }
 
   // Resident slot that holds chunk `ch` (>= n_stream) of the side whose resident part starts at `first`.
   __device__ __forceinline__ int resident_slot(const Cursor first, int ch) const {
@@ -635,6 +638,10 @@ __global__ void __launch_bounds__(kThreads, 1) dvp_row_kernel_resident(const Res
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  DVP_BOUNDS_BEGIN(p.bounds_status);
+  DVP_BOUNDS_SET(n_slot, n_slots);
+  DVP_BOUNDS_SET(V, geo.n_vec);  // this kernel counts a row in 16-byte vectors
+  DVP_BOUNDS_SYNC();
 
   Waiter w = {&ctl->abort, rp.status};
 
@@ -658,6 +665,13 @@ __global__ void __launch_bounds__(kThreads, 1) dvp_row_kernel_resident(const Res
         const int left = geo.n_vec - ch * kSlotVec;
         const uint32_t bytes = (uint32_t)(left < kSlotVec ? left : kSlotVec) * 16u;
         const uint32_t bar = smem_u32(&ctl->full[slot]);
+        // bounds-checking build: a copy outside the slots or past the row is reported and not issued
+        // (the wait for it then runs out and ends the launch, which is reported as well)
+        if (!DVP_IN(slot, n_slot, DVP_OOB_SLOT) ||
+            !DVP_IN((long long)ch * kSlotVec + (long long)bytes / 16 - 1, V, DVP_OOB_GLOBAL)) {
+          cur.advance(ring_slots);
+          return true;
+        }
         mbar_expect_tx(bar, bytes);
         bulk_load(base + (uint32_t)slot * kSlotBytes, row_bytes + (size_t)ch * kSlotBytes, bytes, bar);
         cur.advance(ring_slots);

@@ -148,7 +148,8 @@ __device__ __forceinline__ void drop_below(WarpCand &wc, float tb) {
     const bool stay = valid && widen_bits<TIn>((uint16_t)(e >> 16)) >= tb;
     const uint32_t bal = __ballot_sync(0xffffffffu, stay);
     __syncwarp();  // every lane has read its entry before any lane overwrites one
-    if (stay) wc.list[kept + __popc(bal & ((1u << lane) - 1u))] = e;
+    if (stay && DVP_IN(kept + __popc(bal & ((1u << lane) - 1u)), n_list, DVP_OOB_LIST))
+      wc.list[kept + __popc(bal & ((1u << lane) - 1u))] = e;
     kept += __popc(bal);
   }
   __syncwarp();
@@ -167,8 +168,8 @@ __device__ __forceinline__ void drain(float tb, int n, WarpCand &wc) {
   const int lane = threadIdx.x & 31;
   __syncwarp();  // what other lanes staged is visible
   wc.staged -= n;
-  const bool valid = lane < n;
   const int slot = wc.staged + lane;
+  const bool valid = lane < n && DVP_IN(slot, n_ring, DVP_OOB_RING);
   const uint16_t *vals = reinterpret_cast<const uint16_t *>(wc.ring + 2 * slot);
   uint32_t ord = 0, k = 0;
   if (valid) {
@@ -203,7 +204,8 @@ __device__ __forceinline__ void drain(float tb, int n, WarpCand &wc) {
       const int b = __ffs(k) - 1;
       k &= k - 1;
       const int j = 2 * (b & 7) + (b >> 3);
-      *dst++ = ((uint32_t)vals[j] << 16) | (ord * kElems + (uint32_t)j);
+      if (DVP_IN(dst - wc.list, n_list, DVP_OOB_LIST)) *dst = ((uint32_t)vals[j] << 16) | (ord * kElems + (uint32_t)j);
+      ++dst;
     }
   }
   __syncwarp();  // the slots are free again
@@ -235,14 +237,14 @@ __device__ __forceinline__ void absorb_stage_cs(const TIn *row, int V, const Sta
     const uint32_t bal0 = __ballot_sync(0xffffffffu, hot0), bal1 = __ballot_sync(0xffffffffu, hot1);
     if (bal0 | bal1) {
       const uint32_t below = (1u << lane) - 1u;
-      if (hot0) {
+      if (hot0 && DVP_IN(wc.staged + __popc(bal0 & below), n_ring, DVP_OOB_RING)) {
         const int slot = wc.staged + __popc(bal0 & below);
         wc.ring[2 * slot] = make_uint4(st.g[0].w[0], st.g[0].w[1], st.g[0].w[2], st.g[0].w[3]);
         wc.ring[2 * slot + 1] = make_uint4(st.g[0].w[4], st.g[0].w[5], st.g[0].w[6], st.g[0].w[7]);
         ring_ordinals(wc.ring)[slot] = (uint16_t)(step * 64 + lane);
       }
       wc.staged += __popc(bal0);
-      if (hot1) {
+      if (hot1 && DVP_IN(wc.staged + __popc(bal1 & below), n_ring, DVP_OOB_RING)) {
         const int slot = wc.staged + __popc(bal1 & below);
         wc.ring[2 * slot] = make_uint4(st.g[1].w[0], st.g[1].w[1], st.g[1].w[2], st.g[1].w[3]);
         wc.ring[2 * slot + 1] = make_uint4(st.g[1].w[4], st.g[1].w[5], st.g[1].w[6], st.g[1].w[7]);
@@ -332,6 +334,7 @@ __device__ __forceinline__ FixSum walk_sum(const TIn *row, int V, int n_steps, i
   if (wc.cnt >= 0) {
     const uint32_t pos_a = (uint32_t)position_in_warp(a, kElems);
     for (int i = lane; i < wc.cnt; i += 32) {
+      if (!DVP_IN(i, n_list, DVP_OOB_LIST)) break;
       const uint32_t e = wc.list[i];
       const float x = widen_bits<TIn>((uint16_t)(e >> 16));
       if (x >= tau && x > kNegInf) {  // the fill of a ragged last granule is never a token
@@ -446,7 +449,8 @@ __device__ __forceinline__ void grad_cs(const TIn *row, TGrad *grow, int V, int 
   }
   for (int gi = tid; gi < n_gran; gi += nt) {
     if (gi < n_full) {
-      store_zero_granule<TGrad, kElems>(grow + (size_t)gi * kElems);
+      if (DVP_IN((long long)gi * kElems + kElems - 1, V, DVP_OOB_GLOBAL))
+        store_zero_granule<TGrad, kElems>(grow + (size_t)gi * kElems);
     } else {
       for (int j = 0; j < kElems; ++j) {
         const long long e = (long long)gi * kElems + j;
@@ -464,7 +468,7 @@ __device__ __forceinline__ void grad_cs(const TIn *row, TGrad *grow, int V, int 
     const uint32_t pos = e & 0xffffu, ord = pos / kElems;
     const long long k = ((long long)(ord >> 5) * nt + wbase + (ord & 31u)) * kElems + pos % kElems;
     const float o = pos == pos_a ? g_a : coef * ex2((x - m) * kLog2e);
-    grow[k] = Storage<TGrad>::narrow(o);
+    if (DVP_IN(k, V, DVP_OOB_GLOBAL)) grow[k] = Storage<TGrad>::narrow(o);
   }
 }
 
@@ -490,6 +494,12 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel_cs(const Row
   wc.cap = cap;
 
   constexpr int kElems = Granule<TIn>::kElems;
+  DVP_BOUNDS_BEGIN(p.bounds_status);
+  DVP_BOUNDS_SET(n_gran, (p.V + kElems - 1) / kElems);
+  DVP_BOUNDS_SET(V, p.V);
+  DVP_BOUNDS_SET(n_ring, kRing);
+  DVP_BOUNDS_SET(n_list, cap);
+  DVP_BOUNDS_SYNC();
   const long long t = blockIdx.x;
   const long long id = p.ids ? load_id(p.ids, p.id_is_i32, t) : -1;
   const bool has_id = id >= 0, bad_id = id >= p.V;

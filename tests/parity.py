@@ -11,7 +11,9 @@ Tolerances (stated once, used by every parity test):
     are float32 outputs whose magnitude can reach the hundreds);
   * log_cov = ln Z: 1e-4 absolute, never positive, and the pruned mass 1 - Z
     (the total variation distance of the proof of Prop. 5.5) within 1e-3 relative
-    plus 4e-6 (the float32 sums of up to 2^18 exponentials behind Z);
+    plus 2e-5: Z is a ratio of two float32 sums of up to 2^18 exponentials, whose
+    per-thread chains (a few thousand additions with 64-thread blocks) leave
+    relative errors of up to about 1e-5 on each sum;
   * importance weights (weight_kind): 2e-4 relative (two log-probabilities of
     1e-4 each in the exponent), infinities and NaNs must coincide; rows whose
     ratio lies within 5e-4 relative of a masking bound, where the weight jumps,
@@ -111,13 +113,13 @@ def check_side(got, want, stored, V, label, report):
     comp_want = np.where(want.member == 1, want.sum_safe_x / want.sum_safe, 1.0)
     comp_want = np.where(np.isnan(want.logp), np.nan, comp_want)
     _close(got.comp_mp.cpu(), comp_want, lambda w: 1e-6 + 1e-4 * np.abs(w), f"{label}.comp_mp", ok)
-    # coverage: ln Z within 1e-4, and the pruned mass 1 - Z within 1e-3 relative plus the 4e-6
+    # coverage: ln Z within 1e-4, and the pruned mass 1 - Z within 1e-3 relative plus the 2e-5
     # that float32 sums of up to 2^18 terms leave on Z itself
     lc = got.log_cov.cpu().numpy().astype(np.float64)
     assert (lc <= 0).all(), f"{label}.log_cov must not be positive"
     report[f"{label}_log_cov_err"] = _close(lc, want.log_cov, LOGP_TOL, f"{label}.log_cov", ok)
     pruned_got, pruned_want = -np.expm1(lc[ok]), -np.expm1(want.log_cov[ok])
-    assert (np.abs(pruned_got - pruned_want) <= 1e-3 * pruned_want + 4e-6).all(), f"{label}: 1 - Z"
+    assert (np.abs(pruned_got - pruned_want) <= 1e-3 * pruned_want + 2e-5).all(), f"{label}: 1 - Z"
     if got.mask is not None and want.mask is not None:
         bits = unpack_mask(got.mask, V)
         assert np.array_equal(bits[ok], want.mask[ok]), f"{label}.mask"
