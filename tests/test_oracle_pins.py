@@ -22,6 +22,29 @@ def _rows(rng, T, V, scale=3.0):
     return rng.normal(size=(T, V)) * scale
 
 
+def _safe_set(z: torch.Tensor, rho: float) -> torch.Tensor:
+    """Def. 5.1 as printed, in probability space: k is safe iff pi(k) >= rho max_j pi(j).
+    The inputs of these tests keep every logit away from the threshold, so that this and the
+    logit-space form decide alike (checked)."""
+    with torch.no_grad():
+        pi = torch.softmax(z.detach().to(torch.float64), dim=-1)
+        safe = pi >= rho * pi.max(dim=-1, keepdim=True).values
+        if rho > 0:
+            gap = (torch.log(pi) - torch.log(rho * pi.max(dim=-1, keepdim=True).values)).abs().min()
+            assert gap > 1e-9, "a logit sits on the threshold: the two forms of Def. 5.1 may differ"
+    return safe
+
+
+def _log_pi_mp(z: torch.Tensor, rho: float) -> torch.Tensor:
+    """ln pi^mp of Def. 5.2 by explicit renormalisation: pi^mp(k) = pi(k) / Z on the safe set,
+    Z = sum of pi over the safe set; -inf off it.  Differentiable in z with the set held fixed."""
+    safe = _safe_set(z, rho)
+    pi = torch.softmax(z, dim=-1)
+    cover = (pi * safe).sum(dim=-1, keepdim=True)
+    inside = torch.log(torch.where(safe, pi, torch.ones_like(pi)) / cover)
+    return torch.where(safe, inside, torch.full_like(inside, -math.inf))
+
+
 # --------------------------------------------------------------------------
 # Brute force in probability space (Def. 5.1 and Def. 5.2 as printed), tiny V,
 # extended precision, every token a enumerated.
@@ -121,35 +144,33 @@ def test_invariants(rho):
 
 @pytest.mark.parametrize("rho", [0.2, 1e-2, 1e-4])
 def test_masked_logit_policy_equivalence(rho):
-    """Prop. 5.6 part 1: softmax of the -inf-masked logits is pi^mp.  The mask
-    is built the way App. A builds it (max, + log rho, strict <), by torch."""
+    """Prop. 5.6 part 1: the softmax of logits whose pruned entries are -inf is pi^mp.  The
+    safe set comes from Def. 5.1 in probability space; a library log-softmax of the masked
+    logits and the explicit renormalisation of Def. 5.2 must both give the oracle's value."""
     rng = np.random.default_rng(3)
     z = torch.from_numpy(_rows(rng, 16, 500, scale=3.0))
-    thr = z.max(dim=-1, keepdim=True).values + math.log(rho)
-    z_mp = torch.where(z < thr, torch.tensor(-math.inf, dtype=z.dtype), z)
-    ref = torch.log_softmax(z_mp, dim=-1).numpy()
+    safe = _safe_set(z, rho)
+    ref = torch.log_softmax(z.masked_fill(~safe, -math.inf), dim=-1).numpy()
+    ref2 = _log_pi_mp(z, rho).numpy()
     for a_kind in ("random", "argmax"):
         ids = rng.integers(0, 500, size=16) if a_kind == "random" else z.numpy().argmax(1)
         res = oracle.dvp_rows_f64(z.numpy(), ids, rho, want_mask=True)
-        want = ref[np.arange(16), ids]
-        np.testing.assert_allclose(res.train.logp_mp, want, atol=1e-12, rtol=0)
-        assert np.array_equal(res.train.mask.astype(bool), (z >= thr).numpy())
+        np.testing.assert_allclose(res.train.logp_mp, ref[np.arange(16), ids], atol=1e-12, rtol=0)
+        np.testing.assert_allclose(res.train.logp_mp, ref2[np.arange(16), ids], atol=1e-12, rtol=0)
+        assert np.array_equal(res.train.mask.astype(bool), safe.numpy())
 
 
 @pytest.mark.parametrize("rho", [0.3, 1e-2, 1e-4])
-def test_gradient_matches_autograd_of_masked_log_softmax(rho):
-    """Prop. 5.6 part 2 / Prop. 5.4 with the set fixed (App. A protocol 1)."""
+def test_gradient_matches_autograd_of_the_renormalised_policy(rho):
+    """Prop. 5.4 / Prop. 5.6 part 2 with the set fixed (App. A protocol 1): autograd through
+    pi(a) / Z of Def. 5.2, the safe set entering as a constant."""
     rng = np.random.default_rng(5)
     T, V = 12, 200
     z = torch.from_numpy(_rows(rng, T, V, scale=3.0)).requires_grad_(True)
     g = torch.from_numpy(rng.normal(size=T))
     ids_np = rng.integers(0, V, size=T)
     ids_np[:4] = z.detach().numpy().argmax(1)[:4]
-    with torch.no_grad():
-        thr = z.max(dim=-1, keepdim=True).values + math.log(rho)
-        pruned = z < thr
-    z_mp = torch.where(pruned, torch.tensor(-math.inf, dtype=z.dtype), z)
-    logp = torch.log_softmax(z_mp, dim=-1)[torch.arange(T), torch.from_numpy(ids_np)]
+    logp = _log_pi_mp(z, rho)[torch.arange(T), torch.from_numpy(ids_np)]
     member = torch.isfinite(logp)
     (logp[member] * g[member]).sum().backward()
     res = oracle.dvp_rows_f64(z.detach().numpy(), ids_np, rho, upstream=g.numpy())
@@ -335,10 +356,7 @@ def test_fused_lmhead_matches_autograd_through_the_head():
     ids = rng.integers(0, V, size=T)
     ids[:3] = z.detach().numpy().argmax(1)[:3]
     g = torch.from_numpy(rng.normal(size=T))
-    with torch.no_grad():
-        pruned = z < z.max(dim=-1, keepdim=True).values + math.log(rho)
-    logp = torch.log_softmax(torch.where(pruned, torch.tensor(-math.inf, dtype=z.dtype), z), dim=-1)
-    logp = logp[torch.arange(T), torch.from_numpy(ids)]
+    logp = _log_pi_mp(z, rho)[torch.arange(T), torch.from_numpy(ids)]
     member = torch.isfinite(logp)
     (logp[member] * g[member]).sum().backward()
     bits = lambda x: x.view(torch.int16).numpy().view(np.uint16)
@@ -438,23 +456,34 @@ def test_sequence_level_ratio_is_the_product_of_token_ratios_and_veto_rule():
 
 
 @pytest.mark.parametrize("dt,code", [(torch.bfloat16, oracle.BF16), (torch.float32, oracle.F32)])
-def test_listing_variant_matches_torch_run_of_the_same_steps(dt, code):
-    """App. A taken literally: max, + log(rho) in the logits' dtype, strict <, where
-    with the finite mask value; then a float64 log-softmax and autograd."""
+def test_listing_variant_against_its_closed_form(dt, code):
+    """The finite-mask variant (App. A, Sec. 5.5 "-50.0 in BF16"): pruned tokens keep the
+    probability mass of the mask value.  Stated here as a closed form, not as masked logits:
+    with K the kept set and n the number of pruned tokens,
+        p(a) = e^{z_a} / (sum_K e^{z_k} + n e^{mv}) for a in K,  e^{mv} / (same) otherwise.
+    The threshold is formed in the logits' own type: ln(rho) rounded to it, added to the row
+    maximum in float32, the sum rounded to the type again (an eager tensor expression of that
+    type does exactly this, which the first assertion checks against torch itself)."""
     rng = np.random.default_rng(41)
     T, V, rho, mv = 10, 400, 1e-2, -50.0
     logits = torch.from_numpy((rng.normal(size=(T, V)) * 3).astype(np.float32)).to(dt)
-    with torch.no_grad():
-        threshold = logits.max(dim=-1, keepdim=True).values + math.log(rho)
-        pruned = logits < threshold
-    assert threshold.dtype == dt
+    top = logits.max(dim=-1).values
+    threshold = (top.to(torch.float32) + torch.tensor(math.log(rho)).to(dt).to(torch.float32)).to(dt)[:, None]
+    assert torch.equal(threshold[:, 0], top + math.log(rho)) and threshold.dtype == dt
+    kept = logits >= threshold
+    pruned = ~kept
     z64 = logits.to(torch.float64).requires_grad_(True)
-    masked = torch.where(pruned, torch.tensor(mv, dtype=dt).to(torch.float64), z64)
+    mass_mv = math.exp(torch.tensor(mv, dtype=dt).to(torch.float64).item())
     ids = rng.integers(0, V, size=T)
     ids[:3] = logits.float().numpy().argmax(1)[:3]
     ids[3] = int(np.flatnonzero(pruned[3].numpy())[0])          # a pruned sampled token
     g = torch.from_numpy(rng.normal(size=T))
-    logp = torch.log_softmax(masked, dim=-1)[torch.arange(T), torch.from_numpy(ids)]
+    shift = z64.detach().max(dim=-1, keepdim=True).values       # sums formed relative to the maximum
+    total = (torch.exp(z64 - shift) * kept).sum(dim=-1) + pruned.sum(dim=-1) * mass_mv * torch.exp(-shift[:, 0])
+    picked = z64[torch.arange(T), torch.from_numpy(ids)]
+    own = torch.where(kept[torch.arange(T), torch.from_numpy(ids)], torch.exp(picked - shift[:, 0]),
+                      mass_mv * torch.exp(-shift[:, 0]))
+    logp = torch.log(own / total)
     (logp * g).sum().backward()
     out, grad, thr = oracle.dvp_rows_listing(z64.detach().numpy(), ids, rho, mv, dtype=code, upstream=g.numpy())
     np.testing.assert_array_equal(thr, threshold[:, 0].to(torch.float64).numpy())
@@ -522,9 +551,7 @@ def test_importance_weighted_gradient_matches_autograd_with_a_detached_weight(ki
     ids = torch.from_numpy(ids_np)
 
     def masked_logp(x):
-        with torch.no_grad():
-            pruned = x < x.max(dim=-1, keepdim=True).values + math.log(rho)
-        return torch.log_softmax(torch.where(pruned, torch.tensor(-math.inf, dtype=x.dtype), x), -1)[torch.arange(T), ids]
+        return _log_pi_mp(x, rho)[torch.arange(T), ids]
 
     lt, li = masked_logp(z), masked_logp(zi)
     with torch.no_grad():
@@ -599,9 +626,7 @@ def test_weighted_fused_lmhead_matches_autograd_through_the_head(kind, lo, hi):
     c = torch.from_numpy(rng.normal(size=T))
 
     def masked_logp(x):
-        with torch.no_grad():
-            pruned = x < x.max(dim=-1, keepdim=True).values + math.log(rho)
-        return torch.log_softmax(torch.where(pruned, torch.tensor(-math.inf, dtype=x.dtype), x), -1)[torch.arange(T), idt]
+        return _log_pi_mp(x, rho)[torch.arange(T), idt]
 
     lt, li = masked_logp(z), masked_logp(zi.to(torch.float64))
     with torch.no_grad():
