@@ -271,9 +271,11 @@ int dvp_backward(const dvp_backward_args *args);
  * 16-byte, d_hidden, d_w 32-byte aligned (DVP_ERR_UNSUPPORTED otherwise).
  * Membership is decided on the fp32-accumulated logits, so a token whose logit
  * sits within rounding distance of the threshold may fall on either side of
- * the exact-arithmetic decision.  The gradient panel is held in float16 times
- * a power of two taken from max |upstream|: entries more than about 2^-28
- * below max |upstream| lose relative accuracy.
+ * the exact-arithmetic decision.  The gradient panel is held in float16 as
+ * 2^14 e^{z - max z} on the safe set, the factor of each row (-g / (2^14 s_S))
+ * being applied in float32 afterwards: tokens whose probability is below about
+ * 4e-9 of the row's largest lose relative accuracy, and hidden states beyond
+ * 2047 in magnitude can overflow the float16 copy used for d_w.
  */
 typedef struct {
   uint32_t struct_size;
@@ -406,8 +408,8 @@ int dvp_monitor(const dvp_monitor_args *args);
  *
  * Limit: the workspace the arguments need (dvp_workspace_bytes with the
  * panel_rows this entry uses: pass panel_rows = 128 to that query when you pass 0
- * here, since 0 means up to 4096 there; roughly (2 H + 6 panel_rows) V + 2 H T
- * bytes) must fit in
+ * here, since 0 means up to 4096 there; roughly (2 H + 6 panel_rows) V +
+ * 2 H panel_rows bytes) must fit in
  * DVP_STATIC_WORKSPACE_BYTES, e.g. H = 1024, V = 8192, any T up to a few
  * thousand.  Larger problems return DVP_ERR_WORKSPACE and launch nothing.
  * Other errors are those of dvp_fused_lmhead_forward_backward;

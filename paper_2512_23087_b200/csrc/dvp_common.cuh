@@ -353,7 +353,6 @@ __device__ __forceinline__ float block_reduce_max(float v, float *scratch) {
 struct RowParams {
   const void *train, *infer, *ids;
   const float *upstream;
-  const float *grad_scale;  // optional device scalar multiplied into every upstream gradient
   void *grad;
   long long T, V, ld_train, ld_infer, ld_grad;
   double log_rho;  // ln(rho); -inf for rho = 0
@@ -370,12 +369,6 @@ struct RowParams {
   // ln pi^mp_infer(a) per token, and flags whose DVP_FLAG_IN_TRAIN bit says "a in V'_S"
   const float *given_logp_mp_i;
   const uint8_t *given_flags_i;
-  // 4-byte logits whose row maxima an earlier launch left, in pieces: the maximum of row t is the
-  // largest of given_max[t * given_max_ld + i], i < given_max_n.  The vectorised kernel then needs
-  // one sweep less; the other kernels ignore it.
-  const float *given_max;
-  long long given_max_ld;
-  int given_max_n;
   unsigned int *bounds_status;  // the bounds-checking build's status word; unused otherwise
 };
 

@@ -3,22 +3,25 @@
 // through the head (d_hidden = G W, d_w = G^T hidden) as two more contractions.
 //
 // The [T, V] training logits are never stored: a panel of `panel_rows` tokens
-// lives in the workspace as fp32 logits, is turned into the gradient panel G by
-// the ordinary row kernel, and is consumed by the two gradient contractions
+// lives in the workspace as fp32 logits, is read once by the panel's row pass
+// (dvp_panel.cuh), which leaves the per-token results and the gradient panel up to
+// one factor per row, and that panel is consumed by the two gradient contractions
 // before the next panel overwrites it.
 //
-// G is held in float16 (11-bit significand; bfloat16's 8 bits would miss the
-// 1e-3 gradient tolerance by themselves) times a power of two chosen from
-// max |upstream| so that the panel uses float16's normal range; the inverse
-// power of two is applied in the epilogues of the gradient contractions.
-// tcgen05 kind::f16 needs both operands of one type, so W^T and hidden^T are
-// converted to float16 copies once per call (exact for bfloat16 values in
-// float16's normal range).
+// The panel is held in float16 (11-bit significand; bfloat16's 8 bits would miss
+// the 1e-3 gradient tolerance by themselves): P = 2^14 e^{z - m} on the safe set.
+// The factor per row, -g / (2^14 s_S), multiplies the rows of d_hidden in the
+// contraction's epilogue and, times a power of two chosen from max |upstream|, the
+// hidden rows as they are converted to float16 for the d_w contraction; the inverse
+// power of two is applied in that contraction's epilogue.  tcgen05 kind::f16 needs
+// both operands of one type, so W^T is converted to a float16 copy once per call
+// (exact for bfloat16 values in float16's normal range).
 #include <cmath>
 #include <mutex>
 
 #include "dvp_common.cuh"
 #include "dvp_gemm.cuh"
+#include "dvp_panel.cuh"
 
 namespace dvp {
 
@@ -28,7 +31,7 @@ namespace dvp {
 template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(256)
 transpose_convert_kernel(const TIn *in, long long ld_in, TOut *out, long long ld_out, int R, int C,
-                         int vec_ok) {
+                         int vec_ok, const float *row_scale) {
   __shared__ TOut tile[64][66];
   const int c0 = blockIdx.x * 64, r0 = blockIdx.y * 64;
   const int tid = threadIdx.x;
@@ -37,16 +40,17 @@ transpose_convert_kernel(const TIn *in, long long ld_in, TOut *out, long long ld
   for (int i = 0; i < 2; ++i) {
     const int v = tid + i * 256, r = r0 + (v >> 3), c = c0 + (v & 7) * 8;
     TOut e[8];
+    const float rs = (row_scale && r < R) ? row_scale[r] : 1.f;  // input row r times rs
     if (vec_ok && r < R && c + 8 <= C) {
       const uint4 raw = *reinterpret_cast<const uint4 *>(in + (long long)r * ld_in + c);
       const TIn *x = reinterpret_cast<const TIn *>(&raw);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) e[j] = Storage<TOut>::narrow(Storage<TIn>::widen(x[j]));
+      for (int j = 0; j < 8; ++j) e[j] = Storage<TOut>::narrow(Storage<TIn>::widen(x[j]) * rs);
     } else {
 #pragma unroll
       for (int j = 0; j < 8; ++j)
         e[j] = (r < R && c + j < C)
-                   ? Storage<TOut>::narrow(Storage<TIn>::widen(in[(long long)r * ld_in + c + j]))
+                   ? Storage<TOut>::narrow(Storage<TIn>::widen(in[(long long)r * ld_in + c + j]) * rs)
                    : Storage<TOut>::narrow(0.f);
     }
 #pragma unroll
@@ -72,10 +76,10 @@ transpose_convert_kernel(const TIn *in, long long ld_in, TOut *out, long long ld
 
 template <typename TIn, typename TOut>
 static void launch_transpose(const TIn *in, long long ld_in, TOut *out, long long ld_out, int R, int C,
-                             cudaStream_t s) {
+                             cudaStream_t s, const float *row_scale = nullptr) {
   const int vec_ok = ld_in % 8 == 0 && ld_out % 8 == 0 && (uintptr_t)in % 16 == 0 && (uintptr_t)out % 16 == 0;
   transpose_convert_kernel<TIn, TOut>
-      <<<dim3((C + 63) / 64, (R + 63) / 64), 256, 0, s>>>(in, ld_in, out, ld_out, R, C, vec_ok);
+      <<<dim3((C + 63) / 64, (R + 63) / 64), 256, 0, s>>>(in, ld_in, out, ld_out, R, C, vec_ok, row_scale);
 }
 
 struct FusedScalars {
@@ -128,7 +132,8 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct FusedLayout {
   long long Vp, Tp, panel;
-  size_t off_scalars, off_lpt, off_lpi, off_fli, off_flt, off_wt, off_ht, off_z, off_g, off_rmax, total;
+  size_t off_scalars, off_lpt, off_lpi, off_fli, off_flt, off_wt, off_hs, off_z, off_g, off_rmax, off_rowscale,
+      off_hidscale, off_acoef, off_sort, total;
   long long max_pieces;
 };
 
@@ -157,11 +162,15 @@ bool fused_layout(const dvp_fused_args *a, FusedLayout *L) {
   L->off_fli = take((size_t)a->T);
   L->off_flt = take((size_t)a->T);
   L->off_wt = take((size_t)a->H * L->Vp * 2);
-  L->off_ht = take((size_t)a->H * L->Tp * 2);
+  L->off_hs = take((size_t)a->H * panel * 2);  // the panel's hidden rows, scaled, transposed, float16
   L->off_z = take((size_t)panel * L->Vp * 4);
   L->off_g = take((size_t)panel * L->Vp * 2);
   L->max_pieces = (a->V + gemm::kBN - 1) / gemm::kBN;  // one per tile column of the logits contraction
   L->off_rmax = take((size_t)panel * L->max_pieces * 4);
+  L->off_rowscale = take((size_t)panel * 4);
+  L->off_hidscale = take((size_t)panel * 4);
+  L->off_acoef = take((size_t)panel * 4);
+  L->off_sort = take((size_t)panel::kSortChunk * 8);
   L->total = o;
   return true;
 }
@@ -256,10 +265,14 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
   uint8_t *fli = reinterpret_cast<uint8_t *>(ws + L.off_fli);
   uint8_t *flt = a->flags ? a->flags : reinterpret_cast<uint8_t *>(ws + L.off_flt);
   __half *wt16 = reinterpret_cast<__half *>(ws + L.off_wt);   // [H, Vp]: W^T
-  __half *ht16 = reinterpret_cast<__half *>(ws + L.off_ht);   // [H, Tp]: hidden^T
+  __half *hs16 = reinterpret_cast<__half *>(ws + L.off_hs);   // [H, panel]: the panel's hidden rows, scaled, transposed
   float *z = reinterpret_cast<float *>(ws + L.off_z);         // [panel, Vp] logits
-  __half *g16 = reinterpret_cast<__half *>(ws + L.off_g);     // [panel, Vp] scaled gradient
+  __half *p16 = reinterpret_cast<__half *>(ws + L.off_g);     // [panel, Vp] P = 2^14 e^{z - m} on the safe set
   float *rmax = reinterpret_cast<float *>(ws + L.off_rmax);   // [panel, max_pieces] row maxima of z in pieces
+  float *row_scale = reinterpret_cast<float *>(ws + L.off_rowscale);  // [panel] factor of each row of P
+  float *hid_scale = reinterpret_cast<float *>(ws + L.off_hidscale);  // [panel] the same times a power of two
+  float *a_coef = reinterpret_cast<float *>(ws + L.off_acoef);        // [panel] coefficient of the 1[k = a] term
+  unsigned long long *sorted = reinterpret_cast<unsigned long long *>(ws + L.off_sort);
   const __nv_bfloat16 *hidden = static_cast<const __nv_bfloat16 *>(a->hidden);
   const __nv_bfloat16 *w = static_cast<const __nv_bfloat16 *>(a->w_vocab);
   const int T = (int)a->T, H = (int)a->H, V = (int)a->V;
@@ -269,7 +282,6 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
   const bool weighted = a->weight_kind != DVP_WEIGHT_NONE;
   grad_scale_kernel<<<1, 1024, 0, s>>>(a->upstream, a->T, weighted ? fmaxf(1.f, a->weight_hi) : 1.f, sc);
   launch_transpose<__nv_bfloat16, __half>(w, a->ld_w, wt16, L.Vp, V, H, s);
-  launch_transpose<__nv_bfloat16, __half>(hidden, a->ld_hidden, ht16, L.Tp, T, H, s);
   if (cudaGetLastError() != cudaSuccess) return DVP_ERR_CUDA;
 
   const double log_rho = a->rho > 0.0 ? std::log(a->rho) : -HUGE_VAL;
@@ -294,31 +306,27 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
   for (long long r0 = 0; r0 < a->T; r0 += L.panel, ++panel_index) {
     const int rows = (int)((a->T - r0 < L.panel) ? a->T - r0 : L.panel);
     // logits of the panel: z = hidden[r0 : r0 + rows] x W^T (bf16 operands, fp32 accumulate)
-    // its epilogue also leaves each row's maximum, one piece per tile column: the row kernel
-    // then knows the threshold before it reads the panel and needs one sweep less
+    // its epilogue also leaves each row's maximum, one piece per tile column: the panel's row pass
+    // then knows the threshold before it reads the panel
     cudaError_t e = gemm::launch_gemm_tn(hidden + r0 * a->ld_hidden, a->ld_hidden, w, a->ld_w, z, L.Vp,
                                          rows, V, H, true, 1.f, nullptr, false, &sc->status, sms, s, false,
                                          false, 1, rmax, L.max_pieces);
     if (e != cudaSuccess) return e == cudaErrorInvalidValue ? DVP_ERR_UNSUPPORTED : DVP_ERR_CUDA;
-    // rows of the panel: statistics and G = scale * dLoss/dz in float16
-    RowParams p{};
+    // rows of the panel, one sweep: statistics, and the gradient panel up to a factor per row
+    panel::PanelParams pp{};
+    RowParams &p = pp.row;
     p.train = z;
     p.ids = static_cast<const char *>(a->ids) + r0 * id_bytes;
     p.upstream = a->upstream + r0;
-    p.grad_scale = &sc->scale;
-    p.grad = g16;
     p.T = rows;
     p.V = a->V;
     p.ld_train = L.Vp;
-    p.ld_grad = L.Vp;
     p.log_rho = log_rho;
     p.id_is_i32 = a->id_dtype == DVP_ID_I32;
-    p.given_max = rmax;
-    p.given_max_ld = L.max_pieces;
-    p.given_max_n = (int)L.max_pieces;
     p.out_t = offset_side(a->train, r0, mask_words);
     p.out_t.logp_mp = lpt + r0;
     p.flags = flt + r0;
+    p.bounds_status = bounds_status_word();
     if (weighted) {
       p.weight_kind = (int)a->weight_kind;
       p.weight_lo = a->weight_lo;
@@ -327,20 +335,46 @@ int dvp_fused_lmhead_forward_backward(const dvp_fused_args *a) {
       p.given_logp_mp_i = lpi + r0;
       p.given_flags_i = fli + r0;
     }
-    if (launch_row_kernels(p, DVP_F32, DVP_F16, 0, s) != cudaSuccess) return DVP_ERR_CUDA;
-    // d_hidden[r0 : r0 + rows] = G x W / scale
+    pp.row_max = rmax;
+    pp.row_max_ld = L.max_pieces;
+    pp.row_max_n = (int)L.max_pieces;
+    pp.P = p16;
+    pp.ld_p = L.Vp;
+    pp.row_scale = row_scale;
+    pp.hid_scale = hid_scale;
+    pp.a_coef = a_coef;
+    pp.scale = &sc->scale;
+    panel::dvp_panel_kernel<512, 2><<<(unsigned)rows, 512, 0, s>>>(pp);
+    if (cudaGetLastError() != cudaSuccess) return DVP_ERR_CUDA;
+    // d_hidden[r0 : r0 + rows] = diag(c) P W, the factor applied per row in the epilogue
     // few output tiles and a long K: two K ranges per tile fill the last wave of block pairs
     const long long dh_tiles = ((rows + 255) / 256) * (long long)((H + 255) / 256);
-    e = gemm::launch_gemm_tn(g16, L.Vp, wt16, L.Vp, a->d_hidden + r0 * a->ld_dh, a->ld_dh, rows, H, V,
-                             false, 1.f, &sc->inv_scale, false, &sc->status, sms, s, false, false,
-                             dh_tiles < 8LL * (sms / 2) ? 2 : 1);
+    e = gemm::launch_gemm_tn(p16, L.Vp, wt16, L.Vp, a->d_hidden + r0 * a->ld_dh, a->ld_dh, rows, H, V,
+                             false, 1.f, nullptr, false, &sc->status, sms, s, false, false,
+                             dh_tiles < 8LL * (sms / 2) ? 2 : 1, nullptr, 0, row_scale);
     if (e != cudaSuccess) return e == cudaErrorInvalidValue ? DVP_ERR_UNSUPPORTED : DVP_ERR_CUDA;
-    // d_w (+)= G^T x hidden[r0 : r0 + rows] / scale: G is read as it lies, [rows, V] with V
+    // ... + q_t W[a_t]: the 1[k = a] term in fp32
+    panel::add_sampled_rows_kernel<<<(unsigned)rows, 256, 0, s>>>(
+        a->d_hidden + r0 * a->ld_dh, a->ld_dh, w, a->ld_w, p.ids, p.id_is_i32, a_coef, H);
+    // the panel's hidden rows times their factor (and 2^14 * scale / 512), transposed, in float16
+    launch_transpose<__nv_bfloat16, __half>(hidden + r0 * a->ld_hidden, a->ld_hidden, hs16, L.panel, rows, H, s,
+                                            hid_scale);
+    if (cudaGetLastError() != cudaSuccess) return DVP_ERR_CUDA;
+    // d_w (+)= P^T x (scaled hidden rows) * 512 / (2^14 scale): P is read as it lies, [rows, V] with V
     // contiguous, as the transposed (MN-major) A operand of the contraction
-    e = gemm::launch_gemm_tn(g16, L.Vp, ht16 + r0, L.Tp, a->d_w, a->ld_dw, V, H, rows, false, 1.f,
+    e = gemm::launch_gemm_tn(p16, L.Vp, hs16, L.panel, a->d_w, a->ld_dw, V, H, rows, false, 1.f / 32.f,
                              &sc->inv_scale, panel_index > 0 || a->accumulate_dw != 0, &sc->status, sms,
                              s, false, true);
     if (e != cudaSuccess) return e == cudaErrorInvalidValue ? DVP_ERR_UNSUPPORTED : DVP_ERR_CUDA;
+    // ... + q_t hidden_t into row a_t of d_w: tokens that share a row are added in token order
+    for (int c0 = 0; c0 < rows; c0 += panel::kSortChunk) {
+      const int n = rows - c0 < panel::kSortChunk ? rows - c0 : panel::kSortChunk;
+      const void *ids_c = static_cast<const char *>(p.ids) + (long long)c0 * id_bytes;
+      panel::sort_sampled_ids_kernel<<<1, 1024, 0, s>>>(ids_c, p.id_is_i32, a_coef + c0, n, sorted);
+      panel::add_sampled_hidden_kernel<<<panel::kSortChunk, 256, 0, s>>>(
+          sorted, a_coef + c0, hidden + (r0 + c0) * a->ld_hidden, a->ld_hidden, a->d_w, a->ld_dw, H);
+    }
+    if (cudaGetLastError() != cudaSuccess) return DVP_ERR_CUDA;
   }
 
   if (a->infer_logits) {

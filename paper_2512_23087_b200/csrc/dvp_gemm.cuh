@@ -48,6 +48,7 @@ struct Params {
                            // results are added to C with atomics (C zeroed or accumulated into)
   float *row_max;          // optional (pair kernel, no split, no accumulation): row_max[row * row_max_ld + tn]
   long long row_max_ld;    // = the maximum of row `row` of C over the columns of tile column tn
+  const float *row_scale;  // optional (pair kernel): row `row` of the product is multiplied by row_scale[row]
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -525,7 +526,7 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   } else {
     // ---------------- epilogue (both blocks): own 128 rows of the pair's tile
     const int quarter = warp & 3;
-    const float alpha = p.alpha * (p.alpha_dev ? *p.alpha_dev : 1.f);
+    const float alpha_all = p.alpha * (p.alpha_dev ? *p.alpha_dev : 1.f);
     uint32_t local_tile = 0;
     for (int unit = pair; unit < n_units && !*abort_flag; unit += n_pairs, ++local_tile) {
       const int tile = unit % n_tiles;
@@ -539,6 +540,7 @@ gemm_tn_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       tc_fence_after();
       const int row = tm * kPairBM + (int)rank * kBM + quarter * 32 + lane;
       float *crow = p.C + (long long)row * p.ldc;
+      const float alpha = alpha_all * ((p.row_scale && row < p.M) ? p.row_scale[row] : 1.f);
       float row_hi = -__builtin_huge_valf();  // maximum of what this thread stores of its row
 #pragma unroll 1
       for (int c0 = 0; c0 < kBN; c0 += 32) {
@@ -647,7 +649,7 @@ inline cudaError_t launch_gemm_tn(const void *A, long long lda, const void *B, l
                                   const float *alpha_dev, bool accumulate, int *status, int sm_count,
                                   cudaStream_t stream, bool single_block_tiles = false,
                                   bool a_mn_major = false, int split_k = 1, float *row_max = nullptr,
-                                  long long row_max_ld = 0) {
+                                  long long row_max_ld = 0, const float *row_scale = nullptr) {
   if (M <= 0 || N <= 0 || K <= 0) return cudaSuccess;
   if (lda % 8 || ldb % 8 || ldc % 8 || (uintptr_t)A % 16 || (uintptr_t)B % 16 || (uintptr_t)C % 32)
     return cudaErrorInvalidValue;
@@ -656,8 +658,9 @@ inline cudaError_t launch_gemm_tn(const void *A, long long lda, const void *B, l
   if (single_block_tiles || split_k < 1 || (K + kBK - 1) / kBK < 2 * split_k) split_k = 1;
   // per-tile row maxima are those of the stored values: only where a tile is stored once, whole
   if (row_max && (single_block_tiles || split_k > 1 || accumulate)) return cudaErrorInvalidValue;
+  if (row_scale && single_block_tiles) return cudaErrorInvalidValue;
   Params p{C, ldc, M, N, K, alpha, alpha_dev, accumulate ? 1 : 0, status, a_mn_major ? 1 : 0, split_k,
-           row_max, row_max_ld};
+           row_max, row_max_ld, row_scale};
   if (split_k > 1 && !accumulate) {
     const cudaError_t z = cudaMemset2DAsync(C, (size_t)ldc * 4, 0, (size_t)N * 4, (size_t)M, stream);
     if (z != cudaSuccess) return z;

@@ -451,115 +451,13 @@ __device__ __forceinline__ SumCount row_sweep2(const TIn *row, int V, int a, flo
   return block_reduce_sumcount(sc, scratch);
 }
 
-// One granule of the single statistics sweep of a row whose maximum is known beforehand.
-struct GivenSums {
-  float s_all, s_safe_x;  // sums of e^{z - m}: every token; the safe set without the sampled token
-  int n;                  // |V_S|
-};
-template <typename TIn, int kStage>
-__device__ __forceinline__ void absorb_given(const Granule<TIn> &gr, int slot, int a, float m, float tau,
-                                             GivenSums &acc, uint16_t *bound) {
-  constexpr int kElems = Granule<TIn>::kElems;
-  const int g = slot * (int)blockDim.x + (int)threadIdx.x;
-  const int bi = bound_index<kStage>(slot, threadIdx.x);
-  if (DVP_IN(bi, n_bound, DVP_OOB_BOUND)) bound[bi] = bf16_bits_round_up(gr.max());
-  float x[kElems];
-  gr.get(x);
-  const int ja = a - g * kElems;
-  float all = 0.f;
-#pragma unroll
-  for (int j = 0; j < kElems; ++j) {
-    const float e = ex2((x[j] - m) * kLog2e);  // the fill of a ragged last granule is -inf: e = 0
-    all += e;
-    if (x[j] >= tau && x[j] > kNegInf) {
-      ++acc.n;
-      if (j != ja) acc.s_safe_x += e;
-    }
-  }
-  acc.s_all += all;
-}
-
-// Statistics of a row of 4-byte logits whose maximum an earlier launch left in pieces
-// (RowParams::given_max): with the threshold known before the first logit is read, the full
-// sum, the masked sum and the count come out of one sweep instead of two.
-template <typename TIn, int kStage>
-__device__ __forceinline__ SideStats row_stats_given_max(const TIn *row, int V, int a, const float *pieces,
-                                                         int n_pieces, double log_rho, int mode,
-                                                         float mask_value, uint16_t *bound, float *scratch,
-                                                         uint16_t *hot_smem, HotList &hot, uint32_t *mask_row) {
-  constexpr int kElems = Granule<TIn>::kElems;
-  float mx = kNegInf;
-  for (int i = threadIdx.x; i < n_pieces; i += blockDim.x) mx = fmaxf(mx, pieces[i]);
-  const float m = block_reduce_max(mx, scratch);
-  SideStats st;
-  st.m = m;
-  st.tau = threshold_of<TIn>(m, log_rho, mode);
-  const bool has_a = a >= 0 && a < V;
-  st.z_a = has_a ? Storage<TIn>::widen(row[a]) : 0.f;
-  st.member = has_a && st.z_a >= st.tau;
-  st.e_a = st.member ? ex2((st.z_a - st.m) * kLog2e) : 0.f;
-
-  const int n_full = V / kElems;
-  const int n_gran = (V + kElems - 1) / kElems;
-  const int per_step = kStage * (int)blockDim.x;
-  const int n_steps = (n_gran + per_step - 1) / per_step;
-  GivenSums acc = {0.f, 0.f, 0};
-  if (n_steps > 0) {  // two stages in flight, as in row_sweep1
-    Stage<TIn, kStage> s0, s1;
-    s0.load(row, V, n_full, 0);
-    int step = 0;
-    for (; step + 1 < n_steps; step += 2) {
-      s1.load(row, V, n_full, step + 1);
-#pragma unroll
-      for (int u = 0; u < kStage; ++u) absorb_given<TIn, kStage>(s0.g[u], step * kStage + u, a, m, st.tau, acc, bound);
-      if (step + 2 < n_steps) s0.load(row, V, n_full, step + 2);
-#pragma unroll
-      for (int u = 0; u < kStage; ++u)
-        absorb_given<TIn, kStage>(s1.g[u], (step + 1) * kStage + u, a, m, st.tau, acc, bound);
-    }
-    if (step < n_steps) {
-#pragma unroll
-      for (int u = 0; u < kStage; ++u) absorb_given<TIn, kStage>(s0.g[u], step * kStage + u, a, m, st.tau, acc, bound);
-    }
-  }
-  const SumCount safe = block_reduce_sumcount({acc.s_safe_x, acc.n}, scratch);
-  const SumCount all = block_reduce_sumcount({acc.s_all, 0}, scratch);
-  st.s_x = safe.s;
-  st.n = safe.n;
-  st.lse = (double)m + (double)logf(all.s);
-  st.sum_c = (double)m * (double)kLog2e;
-  st.sum_s = all.s;
-  set_mask_mass(st, V, mode, Storage<TIn>::widen(Storage<TIn>::narrow(mask_value)), has_a);
-  // the list of granules that can hold safe tokens, for the gradient sweep
-  hot = build_hot_list<kStage>(bound, n_steps, bf16_round_down(st.tau), hot_smem);
-  if (mask_row) {
-    const int n_words = (V + 31) / 32;
-    for (int w = threadIdx.x; w < n_words; w += blockDim.x) {
-      uint32_t bits = 0;
-      for (int b = 0; b < 32; ++b) {
-        const long long k = (long long)w * 32 + b;
-        if (k < V && Storage<TIn>::widen(row[k]) >= st.tau) bits |= 1u << b;
-      }
-      mask_row[w] = bits;
-    }
-  }
-  return st;
-}
-
 // Statistics of one side of one row.  `row` is the whole row (V elements); this
-// block sweeps the part [off, off + v_part) of it.  `pieces`: the row's maximum in
-// n_pieces pieces when an earlier launch left it (4-byte logits, one block per row).
+// block sweeps the part [off, off + v_part) of it.
 template <typename TIn, int kStage, int kCluster>
 __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int off, int v_part, int a,
                                                double log_rho, int mode, float mask_value,
                                                uint16_t *bound, float *scratch, float *cl_slots,
-                                               uint16_t *hot_smem, HotList &hot, uint32_t *mask_row,
-                                               const float *pieces = nullptr, int n_pieces = 0) {
-  if constexpr (sizeof(TIn) == 4 && kCluster == 1) {
-    if (pieces)
-      return row_stats_given_max<TIn, kStage>(row, V, a, pieces, n_pieces, log_rho, mode, mask_value, bound,
-                                              scratch, hot_smem, hot, mask_row);
-  }
+                                               uint16_t *hot_smem, HotList &hot, uint32_t *mask_row) {
   const LogSum part = row_sweep1<TIn, kStage>(row + off, v_part, bound, scratch);
   const LogSum all = cluster_reduce_logsum<kCluster>(part, cl_slots);
 
@@ -714,11 +612,10 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
     __syncthreads();  // the bounds and the hot lists are reused for the second matrix
   }
   st = row_stats<TIn, kStage, kCluster>(trow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value, bound,
-                                        scratch, cl_slots, hot_smem, hot, mask_t,
-                                        p.given_max ? p.given_max + t * p.given_max_ld : nullptr, p.given_max_n);
+                                        scratch, cl_slots, hot_smem, hot, mask_t);
 
   if (p.grad) {
-    float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
+    float g = p.upstream[t];
     if constexpr (kWeighted) {
       const float w = p.infer ? row_weight(p, st, si, a >= 0) : row_weight_given(p, st, t, a >= 0);
       if (w == w) g *= w;
@@ -832,7 +729,7 @@ __global__ void dvp_row_kernel_scalar(const RowParams p) {
 
   if (p.grad) {
     TGrad *grow = reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad;
-    float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
+    float g = p.upstream[t];
     if (w == w) g *= w;
     const float s_tot = st.s_x + st.e_a + st.s_mask;
     const bool live = st.live;

@@ -710,7 +710,7 @@ __global__ void __launch_bounds__(kThreads, 1) dvp_row_kernel_resident(const Res
       const TIn *trow = reinterpret_cast<const TIn *>(p.train) + t * p.ld_train;
       const TIn *irow = two_sides ? reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer : nullptr;
       TGrad *grow = p.grad ? reinterpret_cast<TGrad *>(p.grad) + t * p.ld_grad : nullptr;
-      const float g = p.grad ? p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f) : 0.f;
+      const float g = p.grad ? p.upstream[t] : 0.f;
       uint32_t *mask_t = p.out_t.mask ? p.out_t.mask + t * mask_words : nullptr;
       uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * mask_words : nullptr;
       SideStats st, si;

@@ -537,7 +537,7 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel_cs(const Row
                                            run + 1, scratch, mask_row);
     float lp = a >= 0 ? logp_mp_of(s) : nan;
     if (is_train && p.grad) {
-      float g = p.upstream[t] * (p.grad_scale ? *p.grad_scale : 1.f);
+      float g = p.upstream[t];
       if constexpr (kWeighted) {
         float w;
         if (a < 0) {

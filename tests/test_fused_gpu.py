@@ -273,6 +273,19 @@ def test_fused_lmhead_several_panels_and_dw_accumulation():
     assert torch.equal(one.train.count, res.train.count)
 
 
+@pytest.mark.parametrize("panel", [0, 4224, 128])
+def test_fused_lmhead_tokens_that_share_a_sampled_id(panel):
+    """A small vocabulary: most sampled ids occur many times, so the 1[k = a] terms of many tokens
+    meet in the same rows of d_w (they are added in token order: reruns are bit-identical).  A
+    panel of 4224 tokens spans two chunks of that order-fixing step."""
+    T, H, V, rho = 4224, 128, 512, 1e-2
+    batch, res, want, rerun = _run_fused(T, H, V, rho, seed=21, panel_rows=panel)
+    assert len(np.unique(batch.ids.cpu().numpy())) < T // 4
+    _check_fused(batch, rho, res, want, V, rerun=rerun)
+    again = rerun(batch.upstream)
+    assert torch.equal(again.d_w, res.d_w) and torch.equal(again.d_hidden, res.d_hidden)
+
+
 def test_fused_lmhead_full_vocabulary_rows():
     """V = 151,936 with the LM-head statistics of the benchmark configuration."""
     batch, res, want, rerun = _run_fused(256, 1024, 151936, 1e-3, seed=3)
