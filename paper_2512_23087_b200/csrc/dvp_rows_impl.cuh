@@ -42,7 +42,7 @@ struct Granule {
     // granules past the end of the row are legal here (they read as -inf); what the
     // bounds-checking build verifies is that the vector load below stays inside the row
     if (g < 0 || (g < n_full && !DVP_IN((long long)g * kElems + kElems - 1, V, DVP_OOB_GLOBAL))) {
-      DVP_IN(g, n_gran, DVP_OOB_GRANULE);
+      (void)DVP_IN(g, n_gran, DVP_OOB_GRANULE);
       const TIn fill = Storage<TIn>::narrow(kNegInf);
       uint32_t f = 0;
       if constexpr (sizeof(TIn) == 4) {
@@ -255,7 +255,7 @@ __device__ __forceinline__ void granule_grad(const Granule<TIn> &gr, TGrad *grow
   // a granule past the end of the row is legal here (a hot list built for a threshold of -inf
   // names them): nothing of it is stored below.  A negative index is not.
   if (g < 0) {
-    DVP_IN(g, n_gran, DVP_OOB_GRANULE);
+    (void)DVP_IN(g, n_gran, DVP_OOB_GRANULE);
     return;
   }
   if (g < n_full) {
