@@ -45,12 +45,23 @@ NCU_TRAFFIC = {
 }
 
 
-def _kernel_digest() -> str:
+def _kernel_digest(names=("dvp_common.cuh", "dvp_rows_impl.cuh")) -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2512_23087_b200", "csrc")
-    for name in ("dvp_common.cuh", "dvp_rows_impl.cuh"):
+    for name in names:
         h.update(open(os.path.join(csrc, name), "rb").read())
     return h.hexdigest()[:16]
+
+
+# DRAM bytes of the contractions of the fused step (dram__bytes_read.sum + dram__bytes_write.sum of the six
+# gemm_tn_pair_kernel launches of `bench.py --workload c4_fused_lmhead --rows 8192`, H = 4096, V = 151,936,
+# panels of 4096 rows): the first panel's three and a later panel's three (whose d_w contraction also reads
+# the d_w it adds to).  Valid for the sources whose digest is recorded; a step of P panels is taken as the
+# first panel's launches plus P - 1 times the later panel's.
+NCU_TRAFFIC_FUSED = {"digest": "607894dc2e40aeae", "H": 4096, "V": 151936, "panel": 4096,
+                     "first": (4.016951e9 + 2.557340e9) + (13.478416e9 + 0.144871e9) + (4.635654e9 + 2.545532e9),
+                     "later": (3.567931e9 + 2.542042e9) + (13.443569e9 + 0.145225e9) + (7.493283e9 + 2.471862e9)}
+FUSED_SOURCES = ("dvp_gemm.cuh", "dvp_fused.cu", "dvp_panel.cuh")
 
 
 def _peaks():
@@ -568,6 +579,14 @@ def fused_measure(args, rank, world, dev):
         except Exception:
             pass
     achieved = flops / sec / 1e12
+    # DRAM bytes per launch of the contraction kernel, averaged over the step's launches
+    traffic = None
+    rec = NCU_TRAFFIC_FUSED
+    panel = args.panel_rows or min(4096, (T + 127) // 128 * 128)
+    if (rec["digest"] == _kernel_digest(FUSED_SOURCES) and (H, V, panel) == (rec["H"], rec["V"], rec["panel"])
+            and T % panel == 0):
+        n_p = T // panel
+        traffic = (rec["first"] + (n_p - 1) * rec["later"]) / (3 * n_p)
     line = {
         "metric": "fused_lmhead_" + METRIC, "value": tokens / sec, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -582,8 +601,9 @@ def fused_measure(args, rank, world, dev):
                         "per-token results copied back; d_hidden and d_w stay on the device"},
         "gpu_launches": launches,
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                     "frac": achieved / peak, "traffic": None, "peak_kind": f"of {kind}",
-                     "kernel": "gemm_tn_kernel (three contractions per panel)",
+                     "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {kind}",
+                     "kernel": "gemm_tn_pair_kernel (three contractions per panel; traffic = DRAM bytes per launch, "
+                               "mean over the step's launches)",
                      "flops_per_step": flops, "frac_of_burst": achieved / burst,
                      "frac_of_nominal_2250": achieved / 2250.0},
     }
