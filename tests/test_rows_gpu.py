@@ -274,6 +274,28 @@ def test_bf16_logits_with_float32_gradients_at_full_row_length():
               f"{rep16['grad_worst_row_rel_l2']:.2e}, {rep16['grad_frac_rows_above_1e-3']:.3f} of the rows above 1e-3")
 
 
+@pytest.mark.parametrize("grad_dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("sigma,rho", [(1.28, 1e-4), (1.28, 1e-3), (2.2, 1e-4)])
+def test_rows_whose_safe_set_is_most_of_the_vocabulary(sigma, rho, grad_dtype):
+    """bf16 rows of V = 151,936 without a dominant token (the logits a linear head gives for random
+    hidden states): the threshold lies inside the bulk, the safe set holds from a tenth to nearly
+    all of the tokens, most 32-byte pieces of a row are revisited and a warp's list of them
+    overflows, so sweeps 2 and 3 walk every piece instead."""
+    w = W["c2_bf16_fwdbwd"]
+    batch = inputs.make_rows(w, seed=31, device=DEV, T=24)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(32)
+    train = (sigma * torch.randn(24, w.V, device=DEV, generator=g)).to(torch.bfloat16)
+    infer = (train.float() + 0.02 * torch.randn(24, w.V, device=DEV, generator=g)).to(torch.bfloat16)
+    ids = torch.multinomial(torch.softmax(infer.float(), dim=1), 1, generator=g).squeeze(1)  # a ~ softmax(z')
+    batch = dataclasses.replace(batch, train=train, infer=infer, ids=ids)
+    res = _forward(batch, rho, True, grad_dtype=grad_dtype)
+    torch.cuda.synchronize()
+    report, want = parity.check_forward(res, batch, rho, w.V, True)
+    assert report["mean_safe_set_size"] > 0.1 * w.V
+    assert report["grad_zero_rows"] < 24   # sampled tokens below the threshold give zero rows; not all are
+
+
 @pytest.mark.parametrize("name,rho_index", [("c2_bf16_fwdbwd", 0), ("c2_bf16_fwdbwd", 1), ("c3_f32_heavy", 0)])
 def test_full_size_sampled_rows_and_size_free_properties(name, rho_index):
     """The benchmark's own launch at its full size: rows sampled across the
