@@ -69,6 +69,27 @@ struct Granule {
     }
   }
 
+  // Granule `g` of the row's n_full whole granules; any other index reads as -inf.  The row
+  // kernel's sweeps use this one: the elements behind the last whole granule are not theirs (a few
+  // threads take them one by one), so no sweep carries the element-wise code of a ragged granule.
+  __device__ __forceinline__ void load_whole(const TIn *row, int n_full, int g) {
+    if (g < 0 || g >= n_full || !DVP_IN((long long)g * kElems + kElems - 1, V, DVP_OOB_GLOBAL)) {
+      if (g < 0) (void)DVP_IN(g, n_gran, DVP_OOB_GRANULE);
+      const TIn fill = Storage<TIn>::narrow(kNegInf);
+      uint32_t f = 0;
+      if constexpr (sizeof(TIn) == 4) {
+        f = *reinterpret_cast<const uint32_t *>(&fill);
+      } else {
+        const uint32_t h = *reinterpret_cast<const uint16_t *>(&fill);
+        f = h | (h << 16);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) w[i] = f;
+      return;
+    }
+    load(row + (size_t)g * kElems);
+  }
+
   __device__ __forceinline__ void get(float *x) const {
     constexpr int kHalf = kElems / 2;
     Storage<TIn>::unpack(make_uint4(w[0], w[1], w[2], w[3]), x);
@@ -270,10 +291,32 @@ __device__ __forceinline__ void granule_grad(const Granule<TIn> &gr, TGrad *grow
   }
 }
 
+// The same for a whole granule of the row kernel's sweeps (nothing is stored for any other index).
+template <typename TIn, typename TGrad>
+__device__ __forceinline__ void granule_grad_whole(const Granule<TIn> &gr, TGrad *grow, int n_full, int g, int a,
+                                                   float tau, float m, float coef, float g_a) {
+  constexpr int kElems = Granule<TIn>::kElems;
+  if (g < 0 || g >= n_full) {
+    if (g < 0) (void)DVP_IN(g, n_gran, DVP_OOB_GRANULE);
+    return;
+  }
+  float x[kElems], out[kElems];
+  gr.get(x);
+  const int ja = a - g * kElems;
+#pragma unroll
+  for (int j = 0; j < kElems; ++j) {
+    out[j] = x[j] >= tau ? coef * ex2((x[j] - m) * kLog2e) : 0.f;
+    if (j == ja) out[j] = g_a;
+  }
+  if (!DVP_IN((long long)g * kElems + kElems - 1, V, DVP_OOB_GLOBAL)) return;
+  store_granule<TGrad, kElems>(grow + (size_t)g * kElems, out);
+}
+
 // One pipeline stage of sweep 1: kStage granules of this thread.
 template <typename TIn, int kStage>
 struct Stage {
   Granule<TIn> g[kStage];
+  // every granule of the step, the elements of a ragged last granule included
   __device__ __forceinline__ void load(const TIn *row, int V, int n_full, int step) {
     const int g0 = step * kStage * (int)blockDim.x + threadIdx.x;
     if ((step + 1) * kStage * (int)blockDim.x <= n_full &&
@@ -284,6 +327,19 @@ struct Stage {
     } else {
 #pragma unroll
       for (int u = 0; u < kStage; ++u) g[u].load_any(row, V, n_full, g0 + u * (int)blockDim.x);
+    }
+  }
+  // the whole granules of the step only
+  __device__ __forceinline__ void load_whole(const TIn *row, int n_full, int step) {
+    const int g0 = step * kStage * (int)blockDim.x + threadIdx.x;
+    if ((step + 1) * kStage * (int)blockDim.x <= n_full &&
+        DVP_IN(g0 + (kStage - 1) * (int)blockDim.x, n_gran, DVP_OOB_GRANULE)) {
+#pragma unroll
+      for (int u = 0; u < kStage; ++u)
+        g[u].load(row + (size_t)(g0 + u * (int)blockDim.x) * Granule<TIn>::kElems);
+    } else {
+#pragma unroll
+      for (int u = 0; u < kStage; ++u) g[u].load_whole(row, n_full, g0 + u * (int)blockDim.x);
     }
   }
 };
@@ -387,22 +443,35 @@ __device__ __forceinline__ SumCount cluster_reduce_sumcount(SumCount v, float *s
 template <typename TIn, int kStage>
 __device__ __forceinline__ LogSum row_sweep1(const TIn *row, int V, uint16_t *bound, float *scratch) {
   constexpr int kElems = Granule<TIn>::kElems;
-  const int n_full = V / kElems;
-  const int n_gran = (V + kElems - 1) / kElems;
+  const int n_full = V / kElems;  // the sweeps take whole granules; see row_tail
   const int per_step = kStage * (int)blockDim.x;
-  const int n_steps = (n_gran + per_step - 1) / per_step;
+  const int n_steps = (n_full + per_step - 1) / per_step;
   LogSum acc = {kNegInf, kNegInf, 0.f};
   if (n_steps > 0) {  // two stages in flight
     Stage<TIn, kStage> s0, s1;
-    s0.load(row, V, n_full, 0);
+    s0.load_whole(row, n_full, 0);
     int step = 0;
     for (; step + 1 < n_steps; step += 2) {
-      s1.load(row, V, n_full, step + 1);
+      s1.load_whole(row, n_full, step + 1);
       absorb_stage<TIn, kStage>(s0, step, acc, bound);
-      if (step + 2 < n_steps) s0.load(row, V, n_full, step + 2);
+      if (step + 2 < n_steps) s0.load_whole(row, n_full, step + 2);
       absorb_stage<TIn, kStage>(s1, step + 1, acc, bound);
     }
     if (step < n_steps) absorb_stage<TIn, kStage>(s0, step, acc, bound);
+  }
+  // the elements behind the last whole granule, one per thread
+  const int k_tail = n_full * kElems + (int)threadIdx.x;
+  if (k_tail < V) {
+    const float x = Storage<TIn>::widen(row[k_tail]);
+    if (x > kNegInf) {
+      if (x > acc.m) {
+        const float cn = x * kLog2e;
+        acc.s *= ex2(acc.c - cn);
+        acc.m = x;
+        acc.c = cn;
+      }
+      acc.s += ex2(fmaf(x, kLog2e, -acc.c));
+    }
   }
   return block_reduce_logsum(acc, scratch);
 }
@@ -415,11 +484,20 @@ __device__ __forceinline__ SumCount row_sweep2(const TIn *row, int V, int a, flo
                                                uint16_t *hot_smem, HotList &hot) {
   constexpr int kElems = Granule<TIn>::kElems;
   const int n_full = V / kElems;
-  const int n_gran = (V + kElems - 1) / kElems;
   const int per_step = kStage * (int)blockDim.x;
-  const int n_slots = ((n_gran + per_step - 1) / per_step) * kStage;  // granules per thread
+  const int n_slots = ((n_full + per_step - 1) / per_step) * kStage;  // whole granules per thread
   const int tid = threadIdx.x;
   SumCount sc = {0.f, 0};
+  {  // the elements behind the last whole granule, one per thread
+    const int k_tail = n_full * kElems + tid;
+    if (k_tail < V) {
+      const float x = Storage<TIn>::widen(row[k_tail]);
+      if (x >= tau && x > kNegInf) {
+        ++sc.n;
+        if (k_tail != a) sc.s += ex2((x - m) * kLog2e);
+      }
+    }
+  }
   const float tau_b = bf16_round_down(tau);
   hot = build_hot_list<kStage>(bound, n_slots / kStage, tau_b, hot_smem);
   if (hot.fits()) {
@@ -432,8 +510,8 @@ __device__ __forceinline__ SumCount row_sweep2(const TIn *row, int V, int a, flo
       const int g0 = (int)(e0 >> 5) * (int)blockDim.x + wbase + (int)(e0 & 31);
       const int g1 = (int)(e1 >> 5) * (int)blockDim.x + wbase + (int)(e1 & 31);
       Granule<TIn> a0, a1;
-      a0.load_any(row, V, n_full, g0);
-      if (two) a1.load_any(row, V, n_full, g1);
+      a0.load_whole(row, n_full, g0);
+      if (two) a1.load_whole(row, n_full, g1);
       granule_masked_sum<TIn>(a0, g0, a, tau, m, sc);
       if (two) granule_masked_sum<TIn>(a1, g1, a, tau, m, sc);
     }
@@ -443,7 +521,7 @@ __device__ __forceinline__ SumCount row_sweep2(const TIn *row, int V, int a, flo
       if (bf16_bits_to_float(bound[bound_index<kStage>(i, tid)]) >= tau_b) {
         const int g = i * (int)blockDim.x + tid;
         Granule<TIn> gr;
-        gr.load_any(row, V, n_full, g);
+        gr.load_whole(row, n_full, g);
         granule_masked_sum<TIn>(gr, g, a, tau, m, sc);
       }
     }
@@ -503,9 +581,8 @@ __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int
                                          const HotList &hot) {
   constexpr int kElems = Granule<TIn>::kElems;
   const int n_full = V / kElems;
-  const int n_gran = (V + kElems - 1) / kElems;
   const int per_step = kStage * (int)blockDim.x;
-  const int n_slots = ((n_gran + per_step - 1) / per_step) * kStage;
+  const int n_slots = ((n_full + per_step - 1) / per_step) * kStage;
   const int tid = threadIdx.x;
   const float s_tot = st.s_x + st.e_a + st.s_mask;
   // a missing sampled token, or a pruned one under the -inf semantics, has weight zero:
@@ -518,24 +595,27 @@ __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int
   const float tau = live ? st.tau : -kNegInf;  // +inf: nothing passes
   const float tau_b = live ? bf16_round_down(st.tau) : -kNegInf;
 
+  {  // the elements behind the last whole granule, one per thread
+    const int k_tail = n_full * kElems + tid;
+    if (k_tail < V) {
+      const float x = Storage<TIn>::widen(row[k_tail]);
+      float out = x >= tau ? coef * ex2((x - st.m) * kLog2e) : 0.f;
+      if (k_tail == a_live) out = g_a;
+      grow[k_tail] = Storage<TGrad>::narrow(out);
+    }
+  }
   for (int i = 0; i < n_slots; ++i) {
     const int gi = i * (int)blockDim.x + tid;
-    if (gi >= n_gran) break;
+    if (gi >= n_full) break;
     if (!DVP_IN(bound_index<kStage>(i, tid), n_bound, DVP_OOB_BOUND)) break;
     if (bf16_bits_to_float(bound[bound_index<kStage>(i, tid)]) >= tau_b) {
       if (!listed) {
         Granule<TIn> gr;
-        gr.load_any(row, V, n_full, gi);
-        granule_grad<TIn, TGrad>(gr, grow, V, n_full, gi, a_live, tau, st.m, coef, g_a);
+        gr.load_whole(row, n_full, gi);
+        granule_grad_whole<TIn, TGrad>(gr, grow, n_full, gi, a_live, tau, st.m, coef, g_a);
       }
-    } else if (gi < n_full) {
-      if (DVP_IN((long long)gi * kElems + kElems - 1, V, DVP_OOB_GLOBAL))
-        store_zero_granule<TGrad, kElems>(grow + (size_t)gi * kElems);
-    } else {
-      for (int j = 0; j < kElems; ++j) {
-        const long long k = (long long)gi * kElems + j;
-        if (k < V) grow[k] = Storage<TGrad>::narrow(0.f);
-      }
+    } else if (DVP_IN((long long)gi * kElems + kElems - 1, V, DVP_OOB_GLOBAL)) {
+      store_zero_granule<TGrad, kElems>(grow + (size_t)gi * kElems);
     }
   }
   if (listed) {
@@ -548,10 +628,10 @@ __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int
       const int g0 = (int)(e0 >> 5) * (int)blockDim.x + wbase + (int)(e0 & 31);
       const int g1 = (int)(e1 >> 5) * (int)blockDim.x + wbase + (int)(e1 & 31);
       Granule<TIn> a0, a1;
-      a0.load_any(row, V, n_full, g0);
-      if (two) a1.load_any(row, V, n_full, g1);
-      granule_grad<TIn, TGrad>(a0, grow, V, n_full, g0, a_live, tau, st.m, coef, g_a);
-      if (two) granule_grad<TIn, TGrad>(a1, grow, V, n_full, g1, a_live, tau, st.m, coef, g_a);
+      a0.load_whole(row, n_full, g0);
+      if (two) a1.load_whole(row, n_full, g1);
+      granule_grad_whole<TIn, TGrad>(a0, grow, n_full, g0, a_live, tau, st.m, coef, g_a);
+      if (two) granule_grad_whole<TIn, TGrad>(a1, grow, n_full, g1, a_live, tau, st.m, coef, g_a);
     }
   }
 }
