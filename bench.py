@@ -39,9 +39,9 @@ FALLBACK_HBM_GBS = 6650.0
 # from one ncu capture of `bench.py --rows T ...`), keyed by (workload, rho); valid only for
 # the kernel sources whose digest is recorded with it, scaled by rows to the full batch.
 NCU_TRAFFIC = {
-    ("c2_bf16_fwdbwd", 1e-4): {"digest": "2106497854c3e490", "T": 2048, "bytes": 1.658459e9 + 0.610907e9},
-    ("c2_bf16_fwdbwd", 1e-3): {"digest": "2106497854c3e490", "T": 2048, "bytes": 1.351565e9 + 0.604914e9},
-    ("c3_f32_heavy", 1e-4): {"digest": "2106497854c3e490", "T": 1024, "bytes": 2.147959e9 + 1.073491e9},
+    ("c2_bf16_fwdbwd", 1e-4): {"digest": "39dbb5b1cd6d1b57", "T": 2048, "bytes": 1.663427e9 + 0.609676e9},
+    ("c2_bf16_fwdbwd", 1e-3): {"digest": "39dbb5b1cd6d1b57", "T": 2048, "bytes": 1.354367e9 + 0.603508e9},
+    ("c3_f32_heavy", 1e-4): {"digest": "39dbb5b1cd6d1b57", "T": 1024, "bytes": 2.148246e9 + 1.067525e9},
 }
 
 
