@@ -535,7 +535,7 @@ template <typename TIn, int kStage, int kCluster>
 __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int off, int v_part, int a,
                                                double log_rho, int mode, float mask_value,
                                                uint16_t *bound, float *scratch, float *cl_slots,
-                                               uint16_t *hot_smem, HotList &hot, uint32_t *mask_row) {
+                                               uint16_t *hot_smem, HotList &hot) {
   const LogSum part = row_sweep1<TIn, kStage>(row + off, v_part, bound, scratch);
   const LogSum all = cluster_reduce_logsum<kCluster>(part, cl_slots);
 
@@ -558,19 +558,22 @@ __device__ __forceinline__ SideStats row_stats(const TIn *row, int V, int off, i
   st.n = tot.n;
   set_mask_mass(st, V, mode, Storage<TIn>::widen(Storage<TIn>::narrow(mask_value)), has_a);
 
-  // ---- optional packed membership mask (diagnostic output, plain loads)
-  if (mask_row && off == 0) {
-    const int n_words = (V + 31) / 32;
-    for (int w = threadIdx.x; w < n_words; w += blockDim.x) {
-      uint32_t bits = 0;
-      for (int b = 0; b < 32; ++b) {
-        const long long k = (long long)w * 32 + b;
-        if (k < V && Storage<TIn>::widen(row[k]) >= st.tau) bits |= 1u << b;
-      }
-      mask_row[w] = bits;
-    }
-  }
   return st;
+}
+
+// The optional packed membership mask of a row (a diagnostic output): plain loads, one 32-bit word
+// per thread and step.  Called at the end of the kernel, so that its code lies behind the sweeps'.
+template <typename TIn>
+__device__ __forceinline__ void write_mask_row(const TIn *row, int V, float tau, uint32_t *mask_row) {
+  const int n_words = (V + 31) / 32;
+  for (int w = threadIdx.x; w < n_words; w += blockDim.x) {
+    uint32_t bits = 0;
+    for (int b = 0; b < 32; ++b) {
+      const long long k = (long long)w * 32 + b;
+      if (k < V && Storage<TIn>::widen(row[k]) >= tau) bits |= 1u << b;
+    }
+    mask_row[w] = bits;
+  }
 }
 
 // Sweep 3: gradient of g * ln pi^mp(a) over the row.  Granules without a safe
@@ -685,14 +688,13 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
   SideStats st, si;
   if (kWeighted && p.infer) {  // otherwise an earlier launch left the inference side's results
     const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
-    uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
     HotList hot_i;
     si = row_stats<TIn, kStage, kCluster>(irow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value, bound,
-                                          scratch, cl_slots + 8, hot_smem, hot_i, mask_i);
+                                          scratch, cl_slots + 8, hot_smem, hot_i);
     __syncthreads();  // the bounds and the hot lists are reused for the second matrix
   }
   st = row_stats<TIn, kStage, kCluster>(trow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value, bound,
-                                        scratch, cl_slots, hot_smem, hot, mask_t);
+                                        scratch, cl_slots, hot_smem, hot);
 
   if (p.grad) {
     float g = p.upstream[t];
@@ -710,10 +712,9 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
     if (p.infer) {
       __syncthreads();  // the bounds and the hot lists are reused for the second matrix
       const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
-      uint32_t *mask_i = p.out_i.mask ? p.out_i.mask + t * ((p.V + 31) / 32) : nullptr;
-      HotList hot_i;
+        HotList hot_i;
       si = row_stats<TIn, kStage, kCluster>(irow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value,
-                                            bound, scratch, cl_slots + 8, hot_smem, hot_i, mask_i);
+                                            bound, scratch, cl_slots + 8, hot_smem, hot_i);
     }
   }
 
@@ -730,6 +731,12 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
                                                            : log_ratio_of(st.member, si.member, lt, li);
     }
     if (p.flags) p.flags[t] = flags;
+  }
+  if (off == 0) {  // the first block of a row's cluster writes the row's masks
+    if (mask_t) write_mask_row<TIn>(trow, V, st.tau, mask_t);
+    if (p.infer && p.out_i.mask)
+      write_mask_row<TIn>(reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer, V, si.tau,
+                          p.out_i.mask + t * ((p.V + 31) / 32));
   }
   // no block may leave while another one can still read its exchange slots
   if constexpr (kCluster > 1) cluster_sync_all();
