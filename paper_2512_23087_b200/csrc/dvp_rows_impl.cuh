@@ -712,7 +712,7 @@ __global__ void __launch_bounds__(kThreads, kBlocks) dvp_row_kernel(const RowPar
     if (p.infer) {
       __syncthreads();  // the bounds and the hot lists are reused for the second matrix
       const TIn *irow = reinterpret_cast<const TIn *>(p.infer) + t * p.ld_infer;
-        HotList hot_i;
+      HotList hot_i;
       si = row_stats<TIn, kStage, kCluster>(irow, V, off, v_part, a, p.log_rho, p.mode, p.mask_value,
                                             bound, scratch, cl_slots + 8, hot_smem, hot_i);
     }
