@@ -39,9 +39,9 @@ FALLBACK_HBM_GBS = 6650.0
 # from one ncu capture of `bench.py --rows T ...`), keyed by (workload, rho); valid only for
 # the kernel sources whose digest is recorded with it, scaled by rows to the full batch.
 NCU_TRAFFIC = {
-    ("c2_bf16_fwdbwd", 1e-4): {"digest": "39dbb5b1cd6d1b57", "T": 2048, "bytes": 1.663427e9 + 0.609676e9},
-    ("c2_bf16_fwdbwd", 1e-3): {"digest": "39dbb5b1cd6d1b57", "T": 2048, "bytes": 1.354367e9 + 0.603508e9},
-    ("c3_f32_heavy", 1e-4): {"digest": "39dbb5b1cd6d1b57", "T": 1024, "bytes": 2.148246e9 + 1.067525e9},
+    ("c2_bf16_fwdbwd", 1e-4): {"digest": "77c48103593e9e9c", "T": 2048, "bytes": 1.664036e9 + 0.609036e9},
+    ("c2_bf16_fwdbwd", 1e-3): {"digest": "77c48103593e9e9c", "T": 2048, "bytes": 1.355791e9 + 0.602884e9},
+    ("c3_f32_heavy", 1e-4): {"digest": "77c48103593e9e9c", "T": 1024, "bytes": 2.148025e9 + 1.067222e9},
 }
 
 
