@@ -126,45 +126,44 @@ __global__ void __launch_bounds__(256, 3) dvp_monitor_kernel(const MonitorParams
   DVP_BOUNDS_SYNC();
   Moments a = {kNegInf, kNegInf, 0.f, 0.f, 0.f}, b = a;
   if constexpr (kVector) {
-    const int n_full = V / kElems, n_gran = (V + kElems - 1) / kElems;
-    for (int g = threadIdx.x; g < n_gran; g += 2 * blockDim.x) {
+    // whole granules in the loop; the elements behind the last whole granule one per thread after
+    // it, so that the loop carries no element-wise code for a ragged granule
+    const int n_full = V / kElems;
+    for (int g = threadIdx.x; g < n_full; g += 2 * blockDim.x) {
       const int g2 = g + blockDim.x;
       Granule<TIn> ta, ia, tb, ib;  // two granules of each row in flight
-      ta.load_any(zt, V, n_full, g);
-      ia.load_any(zi, V, n_full, g);
-      const bool second = g2 < n_gran;
+      if (!DVP_IN((long long)g * kElems + kElems - 1, V, DVP_OOB_GLOBAL)) break;
+      ta.load(zt + (size_t)g * kElems);
+      ia.load(zi + (size_t)g * kElems);
+      const bool second = g2 < n_full && DVP_IN((long long)g2 * kElems + kElems - 1, V, DVP_OOB_GLOBAL);
       if (second) {
-        tb.load_any(zt, V, n_full, g2);
-        ib.load_any(zi, V, n_full, g2);
+        tb.load(zt + (size_t)g2 * kElems);
+        ib.load(zi + (size_t)g2 * kElems);
       }
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         if (h == 1 && !second) break;
         const Granule<TIn> &gt = h ? tb : ta, &gi = h ? ib : ia;
-        const int gg = h ? g2 : g;
         float x[kElems], y[kElems];
         gt.get(x);
         gi.get(y);
         raise(a, gt.max());
         raise(b, gi.max());
-        if (gg < n_full) {
 #pragma unroll
-          for (int j = 0; j < kElems; ++j) {
-            const float d = y[j] - x[j];
-            absorb(a, x[j], d);
-            absorb(b, y[j], d);
-          }
-        } else {  // the ragged last granule: elements past V were filled with -inf
-#pragma unroll
-          for (int j = 0; j < kElems; ++j) {
-            if ((long long)gg * kElems + j < V) {
-              const float d = y[j] - x[j];
-              absorb(a, x[j], d);
-              absorb(b, y[j], d);
-            }
-          }
+        for (int j = 0; j < kElems; ++j) {
+          const float d = y[j] - x[j];
+          absorb(a, x[j], d);
+          absorb(b, y[j], d);
         }
       }
+    }
+    const int k_tail = n_full * kElems + (int)threadIdx.x;
+    if (k_tail < V) {
+      const float x = Storage<TIn>::widen(zt[k_tail]), y = Storage<TIn>::widen(zi[k_tail]);
+      raise(a, x);
+      raise(b, y);
+      absorb(a, x, y - x);
+      absorb(b, y, y - x);
     }
   } else {
     float mt = kNegInf, mi = kNegInf;
