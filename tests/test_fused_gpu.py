@@ -229,7 +229,10 @@ def _run_fused(T, H, V, rho, seed, weight=None, **kw):
 
 
 @pytest.mark.parametrize("T,H,V,rho", [(200, 256, 3000, 1e-3), (64, 128, 1000, 1e-2), (130, 512, 5008, 1e-4),
-                                       (128, 4096, 4096, 1e-3)])
+                                       (128, 4096, 4096, 1e-3),
+                                       # vocabularies that end inside a 32-byte piece of the fp32 panel and
+                                       # inside a 16-element block of the contractions' tiles
+                                       (96, 128, 1003, 1e-2), (140, 256, 4099, 1e-3), (70, 64, 7, 1e-1)])
 def test_fused_lmhead_small(T, H, V, rho):
     batch, res, want, rerun = _run_fused(T, H, V, rho, seed=T)
     _check_fused(batch, rho, res, want, V, rerun=rerun)
