@@ -686,6 +686,60 @@ def dry_run_ranks(args):
         dist.destroy_process_group()
 
 
+def run_row_classes(args):
+    """Where the time of a row workload goes: batches made of copies of ONE row each, the rows taken at
+    percentiles of the number of 32-byte granules that hold a safe token (every copy has its own memory),
+    timed like the headline.  One JSON line; a diagnostic, not the benchmark."""
+    import math
+    import torch
+    from paper_2512_23087_b200 import binding, inputs
+    w = inputs.WORKLOADS[args.workload]
+    rho = args.rho if args.rho is not None else w.rhos[0]
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    pool, T, V = 2048, args.rows or 8192, w.V
+    b = inputs.make_rows(w, seed=0, device=dev, T=pool)
+    elem = b.train.element_size()
+    per_granule = 32 // elem
+    z = b.train.float()
+    tau = z.max(dim=1).values + math.log(rho)
+    hot = (z.view(pool, -1, per_granule).max(dim=2).values >= tau[:, None]).sum(dim=1)
+    safe = (z >= tau[:, None]).sum(dim=1)
+    del z
+    order = torch.argsort(hot)
+    grad_dtype = torch.float32 if w.dtype == "f32" else b.train.dtype
+    out = []
+    for pct in (1, 25, 50, 75, 90, 95, 99, 100):
+        i = int(order[min(pool - 1, pool * pct // 100)])
+        train = b.train[i:i + 1].expand(T, V).contiguous()
+        infer = b.infer[i:i + 1].expand(T, V).contiguous()
+        ids = b.ids[i:i + 1].expand(T).contiguous()
+        up = b.upstream[i:i + 1].expand(T).contiguous() if w.backward else None
+        res = None
+        for _ in range(max(3, args.warmup)):
+            res = binding.dvp_forward(train, ids, rho, infer_logits=infer, upstream=up, grad_dtype=grad_dtype,
+                                      launch_hint=args.launch_hint, out=res)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            binding.dvp_forward(train, ids, rho, infer_logits=infer, upstream=up, grad_dtype=grad_dtype,
+                                launch_hint=args.launch_hint, out=res)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.steps
+        alg = (2 * elem + (res.grad_train.element_size() if w.backward else 0)) * T * V
+        out.append({"percentile": pct, "hot_granules": int(hot[i]), "safe_tokens": int(safe[i]),
+                    "ms_per_step": ms, "achieved_gbs": alg / ms / 1e6})
+        del train, infer, res
+    peak, kind = _peaks()
+    for o in out:
+        o["frac"] = o["achieved_gbs"] / peak
+    print(json.dumps({"row_classes": out, "workload": w.name, "rho": rho, "T": T, "V": V, "granules_per_row":
+                      (V + per_granule - 1) // per_granule, "steps": args.steps, "peak": peak,
+                      "peak_kind": f"of {kind}"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -702,6 +756,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--panel-rows", type=int, default=0, help="fused workload: tokens per panel")
     ap.add_argument("--no-extras", action="store_true", help="headline workload only")
+    ap.add_argument("--row-classes", action="store_true",
+                    help="time batches of copies of one row each, by percentile of revisited granules (a diagnostic)")
     ap.add_argument("--dry-run-ranks", action="store_true",
                     help="ranks only rendezvous (gloo, no GPU) and reduce a number: checks the launch path")
     args = ap.parse_args()
@@ -709,6 +765,8 @@ def main():
         raise SystemExit(spawn_ranks(args.gpus))
     if args.dry_run_ranks:
         return dry_run_ranks(args)
+    if args.row_classes:
+        return run_row_classes(args)
     if args.workload == "c4_fused_lmhead":
         if args.impl == "reference":
             if int(os.environ.get("RANK", "0")) == 0:
