@@ -516,14 +516,18 @@ __device__ __forceinline__ SumCount row_sweep2(const TIn *row, int V, int a, flo
       if (two) granule_masked_sum<TIn>(a1, g1, a, tau, m, sc);
     }
   } else {
-    for (int i = 0; i < n_slots; ++i) {
-      if (!DVP_IN(bound_index<kStage>(i, tid), n_bound, DVP_OOB_BOUND)) break;
-      if (bf16_bits_to_float(bound[bound_index<kStage>(i, tid)]) >= tau_b) {
-        const int g = i * (int)blockDim.x + tid;
-        Granule<TIn> gr;
-        gr.load_whole(row, n_full, g);
-        granule_masked_sum<TIn>(gr, g, a, tau, m, sc);
-      }
+    // a dense safe set: all of the thread's granules, a step's two at a time (both loads before either is used)
+    static_assert(kStage == 2, "a step's two bounds are neighbours");
+    for (int i = 0; i < n_slots; i += 2) {
+      if (!DVP_IN(bound_index<kStage>(i + 1, tid), n_bound, DVP_OOB_BOUND)) break;
+      const bool hot0 = bf16_bits_to_float(bound[bound_index<kStage>(i, tid)]) >= tau_b;
+      const bool hot1 = bf16_bits_to_float(bound[bound_index<kStage>(i + 1, tid)]) >= tau_b;
+      const int g0 = i * (int)blockDim.x + tid, g1 = g0 + (int)blockDim.x;
+      Granule<TIn> a0, a1;
+      if (hot0) a0.load_whole(row, n_full, g0);
+      if (hot1) a1.load_whole(row, n_full, g1);
+      if (hot0) granule_masked_sum<TIn>(a0, g0, a, tau, m, sc);
+      if (hot1) granule_masked_sum<TIn>(a1, g1, a, tau, m, sc);
     }
   }
   return block_reduce_sumcount(sc, scratch);
