@@ -616,13 +616,24 @@ __device__ __forceinline__ void row_grad(const TIn *row, TGrad *grow, int V, int
     if (gi >= n_full) break;
     if (!DVP_IN(bound_index<kStage>(i, tid), n_bound, DVP_OOB_BOUND)) break;
     if (bf16_bits_to_float(bound[bound_index<kStage>(i, tid)]) >= tau_b) {
-      if (!listed) {
-        Granule<TIn> gr;
-        gr.load_whole(row, n_full, gi);
-        granule_grad_whole<TIn, TGrad>(gr, grow, n_full, gi, a_live, tau, st.m, coef, g_a);
-      }
+      // a granule that can hold safe tokens: written below
     } else if (DVP_IN((long long)gi * kElems + kElems - 1, V, DVP_OOB_GLOBAL)) {
       store_zero_granule<TGrad, kElems>(grow + (size_t)gi * kElems);
+    }
+  }
+  if (live && !listed) {
+    // a dense safe set: all of the thread's hot granules, a step's two at a time (both loads before either is used)
+    static_assert(kStage == 2, "a step's two bounds are neighbours");
+    for (int i = 0; i < n_slots; i += 2) {
+      if (!DVP_IN(bound_index<kStage>(i + 1, tid), n_bound, DVP_OOB_BOUND)) break;
+      const int g0 = i * (int)blockDim.x + tid, g1 = g0 + (int)blockDim.x;
+      const bool hot0 = g0 < n_full && bf16_bits_to_float(bound[bound_index<kStage>(i, tid)]) >= tau_b;
+      const bool hot1 = g1 < n_full && bf16_bits_to_float(bound[bound_index<kStage>(i + 1, tid)]) >= tau_b;
+      Granule<TIn> a0, a1;
+      if (hot0) a0.load_whole(row, n_full, g0);
+      if (hot1) a1.load_whole(row, n_full, g1);
+      if (hot0) granule_grad_whole<TIn, TGrad>(a0, grow, n_full, g0, a_live, tau, st.m, coef, g_a);
+      if (hot1) granule_grad_whole<TIn, TGrad>(a1, grow, n_full, g1, a_live, tau, st.m, coef, g_a);
     }
   }
   if (listed) {
