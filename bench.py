@@ -39,9 +39,9 @@ FALLBACK_HBM_GBS = 6650.0
 # from one ncu capture of `bench.py --rows T ...`), keyed by (workload, rho); valid only for
 # the kernel sources whose digest is recorded with it, scaled by rows to the full batch.
 NCU_TRAFFIC = {
-    ("c2_bf16_fwdbwd", 1e-4): {"digest": "77c48103593e9e9c", "T": 2048, "bytes": 1.664036e9 + 0.609036e9},
-    ("c2_bf16_fwdbwd", 1e-3): {"digest": "77c48103593e9e9c", "T": 2048, "bytes": 1.355791e9 + 0.602884e9},
-    ("c3_f32_heavy", 1e-4): {"digest": "77c48103593e9e9c", "T": 1024, "bytes": 2.148025e9 + 1.067222e9},
+    ("c2_bf16_fwdbwd", 1e-4): {"digest": "47f036696d37ae2e", "T": 2048, "bytes": 1.663986e9 + 0.608635e9},
+    ("c2_bf16_fwdbwd", 1e-3): {"digest": "47f036696d37ae2e", "T": 2048, "bytes": 1.354420e9 + 0.603881e9},
+    ("c3_f32_heavy", 1e-4): {"digest": "47f036696d37ae2e", "T": 1024, "bytes": 2.148133e9 + 1.068105e9},
 }
 
 
